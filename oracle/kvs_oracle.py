@@ -1,0 +1,350 @@
+"""CPU fp64 oracle for eviction-masked causal attention (TEST INFRASTRUCTURE).
+
+This file is the slow, plain statement of what the CUDA path must compute.  It
+is imported only by the tests, by the smoke check and by the benchmark's CPU
+baseline leg; the library never calls it, and it shares no code with the CUDA
+sources.
+
+What it states, and where that comes from:
+
+* Mask.  Sec. 2 ("KV-streams" paragraph) and the caption of Fig. 2 say that the
+  trainer processes ONE continuous trace and that a custom attention mask
+  blocks attention to the span the inference engine deleted, so that one
+  forward pass reproduces the rollout's evictions.  Encoded per key as an
+  eviction step: query ``i`` may read key ``j`` iff ``j <= i < evict_at[j]``.
+  Positions are not reset (Sec. 2: retained entries keep their ``(k_i, v_i)``),
+  so q and k are used as given.
+* ``dense_*``: softmax attention under that boolean mask, written out from the
+  definition, with its analytic gradients.
+* ``replay_*``: the rollout itself (Sec. 1 and Sec. 2: KV entries are evicted
+  directly in the engine's cache).  A cache of rows is kept; before token ``i``
+  is processed every row whose eviction step is ``i`` is physically removed;
+  token ``i`` is appended; ``q_i`` attends over exactly the rows present.  No
+  mask is ever consulted.  Agreement of the two routes is the check that the
+  mask above is the one that reproduces eviction.
+* Tile classes: the min/max rule per 128x128 tile and, independently, a brute
+  force classification from the dense boolean mask.
+
+Everything is fp64 on inputs that were already rounded to bf16 by the caller.
+Pins (tests/test_oracle_pins.py): two-route agreement, no-eviction == plain
+causal attention (torch's CPU scaled_dot_product_attention in fp64), softmax
+rows summing to one, central finite differences for dQ/dK/dV, zero-query
+closed forms (exp(LSE) = live-key count, values printed in tests/golden),
+evict-after-one-step closed form, exact integer pair and tile counts.
+No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+INF = 2**31 - 1
+BLOCK = 128
+EMPTY, PARTIAL, FULL = 0, 1, 2
+
+
+# --------------------------------------------------------------------------
+# mask
+# --------------------------------------------------------------------------
+def allowed(evict_at: np.ndarray) -> np.ndarray:
+    """Boolean [T, T]: allowed[i, j] = (j <= i) and (i < evict_at[j])."""
+    ev = np.asarray(evict_at, dtype=np.int64)
+    T = ev.shape[0]
+    i = np.arange(T, dtype=np.int64)[:, None]
+    j = np.arange(T, dtype=np.int64)[None, :]
+    return (j <= i) & (i < ev[None, :])
+
+
+def check_evict_at(evict_at: np.ndarray) -> None:
+    """Precondition: every key is visible at least to its own query."""
+    ev = np.asarray(evict_at, dtype=np.int64)
+    j = np.arange(ev.shape[0], dtype=np.int64)
+    if np.any(ev <= j):
+        raise ValueError("evict_at[j] <= j for some key")
+
+
+# --------------------------------------------------------------------------
+# dense masked attention, one trace
+# --------------------------------------------------------------------------
+def dense_fwd(q, k, v, evict_at, scale):
+    """q [T,Hq,d], k,v [T,Hkv,d] (any float dtype; widened to fp64).
+    Returns out [T,Hq,d] fp64, lse [Hq,T] fp64 (natural log, scale included)."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    check_evict_at(evict_at)
+    A = allowed(evict_at)
+    out = np.zeros((T, Hq, d))
+    lse = np.zeros((Hq, T))
+    for h in range(Hq):
+        g = h // G
+        S = scale * (q[:, h, :] @ k[:, g, :].T)
+        S = np.where(A, S, -np.inf)
+        m = S.max(axis=1, keepdims=True)
+        E = np.exp(S - m)
+        l = E.sum(axis=1, keepdims=True)
+        P = E / l
+        out[:, h, :] = P @ v[:, g, :]
+        lse[h, :] = (m + np.log(l))[:, 0]
+    return out, lse
+
+
+def dense_bwd(q, k, v, dout, evict_at, scale):
+    """Analytic gradients of sum(out * dout) w.r.t. q, k, v.
+    Returns dq [T,Hq,d], dk, dv [T,Hkv,d] (fp64)."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    dout = np.asarray(dout, dtype=np.float64)
+    T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    A = allowed(evict_at)
+    dq = np.zeros_like(q)
+    dk = np.zeros_like(k)
+    dv = np.zeros_like(v)
+    for h in range(Hq):
+        g = h // G
+        S = scale * (q[:, h, :] @ k[:, g, :].T)
+        S = np.where(A, S, -np.inf)
+        m = S.max(axis=1, keepdims=True)
+        E = np.exp(S - m)
+        P = E / E.sum(axis=1, keepdims=True)
+        O = P @ v[:, g, :]
+        dP = dout[:, h, :] @ v[:, g, :].T
+        D = (dout[:, h, :] * O).sum(axis=1, keepdims=True)
+        dS = P * (dP - D)
+        dq[:, h, :] = scale * (dS @ k[:, g, :])
+        dk[:, g, :] += scale * (dS.T @ q[:, h, :])
+        dv[:, g, :] += P.T @ dout[:, h, :]
+    return dq, dk, dv
+
+
+# --------------------------------------------------------------------------
+# incremental replay with physical eviction, one trace
+# --------------------------------------------------------------------------
+def replay_fwd_bwd(q, k, v, dout, evict_at, scale, removal="ordered"):
+    """Replays the rollout token by token.  The cache is a Python list of
+    original key indices; rows leave it for good at their eviction step.
+
+    removal: "ordered" keeps the surviving rows in order, "swap" moves the
+    last row into the hole (row order must not matter).
+    Returns out, lse, dq, dk, dv, cache_sizes (int array, rows present when
+    token i attends).  ``dout`` may be None (then the gradients are None)."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    ev = np.asarray(evict_at, dtype=np.int64)
+    check_evict_at(ev)
+    # keys bucketed by the step at which the engine drops them
+    leaving = {}
+    for j in range(T):
+        if ev[j] < T:
+            leaving.setdefault(int(ev[j]), []).append(j)
+    out = np.zeros((T, Hq, d))
+    lse = np.zeros((Hq, T))
+    sizes = np.zeros(T, dtype=np.int64)
+    want_grad = dout is not None
+    if want_grad:
+        dout = np.asarray(dout, dtype=np.float64)
+        dq = np.zeros_like(q)
+        dk = np.zeros_like(k)
+        dv = np.zeros_like(v)
+    cache = []          # original indices of the rows present
+    where = {}          # original index -> slot in `cache`
+    for i in range(T):
+        for j in leaving.get(i, ()):
+            slot = where.pop(j)
+            if removal == "swap":
+                last = cache.pop()
+                if last != j:
+                    cache[slot] = last
+                    where[last] = slot
+            else:
+                del cache[slot]
+                for s in range(slot, len(cache)):
+                    where[cache[s]] = s
+        where[i] = len(cache)
+        cache.append(i)
+        rows = np.asarray(cache, dtype=np.int64)
+        sizes[i] = rows.shape[0]
+        for h in range(Hq):
+            g = h // G
+            Kc = k[rows, g, :]
+            Vc = v[rows, g, :]
+            s = scale * (Kc @ q[i, h, :])
+            m = s.max()
+            e = np.exp(s - m)
+            l = e.sum()
+            p = e / l
+            o = p @ Vc
+            out[i, h, :] = o
+            lse[h, i] = m + np.log(l)
+            if want_grad:
+                do = dout[i, h, :]
+                dp = Vc @ do
+                ds = p * (dp - do @ o)
+                dq[i, h, :] = scale * (ds @ Kc)
+                np.add.at(dk[:, g, :], rows, scale * np.outer(ds, q[i, h, :]))
+                np.add.at(dv[:, g, :], rows, np.outer(p, do))
+    if want_grad:
+        return out, lse, dq, dk, dv, sizes
+    return out, lse, None, None, None, sizes
+
+
+# --------------------------------------------------------------------------
+# packed (varlen) wrappers
+# --------------------------------------------------------------------------
+def varlen_fwd(q, k, v, evict_at, cu_seqlens, scale):
+    q = np.asarray(q, dtype=np.float64)
+    Ttot, Hq, d = q.shape
+    out = np.zeros((Ttot, Hq, d))
+    lse = np.zeros((Hq, Ttot))
+    for b in range(len(cu_seqlens) - 1):
+        a, e = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        if e == a:
+            continue
+        o, l = dense_fwd(q[a:e], k[a:e], v[a:e], evict_at[a:e], scale)
+        out[a:e] = o
+        lse[:, a:e] = l
+    return out, lse
+
+
+def varlen_bwd(q, k, v, dout, evict_at, cu_seqlens, scale):
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    dq = np.zeros_like(q)
+    dk = np.zeros_like(k)
+    dv = np.zeros_like(k)
+    for b in range(len(cu_seqlens) - 1):
+        a, e = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        if e == a:
+            continue
+        x, y, z = dense_bwd(q[a:e], k[a:e], v[a:e], dout[a:e], evict_at[a:e], scale)
+        dq[a:e], dk[a:e], dv[a:e] = x, y, z
+    return dq, dk, dv
+
+
+# --------------------------------------------------------------------------
+# single rows / single key blocks of a long trace (for full-size sampling)
+# --------------------------------------------------------------------------
+def row_fwd(q_i, k, v, evict_at, i, scale):
+    """One query row ``i`` of one head.  q_i [d]; k, v [T, d] of its KV head.
+    Returns o [d], lse (float), visible key indices, p over them."""
+    ev = np.asarray(evict_at[: i + 1], dtype=np.int64)
+    vis = np.nonzero(ev > i)[0]
+    Kc = np.asarray(k[vis], dtype=np.float64)
+    Vc = np.asarray(v[vis], dtype=np.float64)
+    s = scale * (Kc @ np.asarray(q_i, dtype=np.float64))
+    m = s.max()
+    e = np.exp(s - m)
+    l = e.sum()
+    p = e / l
+    return p @ Vc, m + np.log(l), vis, p
+
+
+def row_fwd_bwd(q_i, k, v, do_i, evict_at, i, scale):
+    """As row_fwd, plus dq_i [d] and this row's contributions (vis, dk_rows, dv_rows)."""
+    o, lse, vis, p = row_fwd(q_i, k, v, evict_at, i, scale)
+    Kc = np.asarray(k[vis], dtype=np.float64)
+    Vc = np.asarray(v[vis], dtype=np.float64)
+    do = np.asarray(do_i, dtype=np.float64)
+    dp = Vc @ do
+    ds = p * (dp - do @ o)
+    dq = scale * (ds @ Kc)
+    return o, lse, dq, vis, scale * np.outer(ds, np.asarray(q_i, dtype=np.float64)), np.outer(p, do)
+
+
+def key_block_dkdv(q, k, v, dout, evict_at, j0, j1, g, G, scale):
+    """dK, dV for keys [j0, j1) of KV head ``g`` of one trace: every query row
+    that can see any of those keys is evaluated in full (its softmax needs all
+    of its visible keys).  q, dout [T,Hq,d]; k, v [T,Hkv,d].
+    Returns dk [j1-j0, d], dv [j1-j0, d]."""
+    ev = np.asarray(evict_at, dtype=np.int64)
+    T = ev.shape[0]
+    last = int(min(T, ev[j0:j1].max()))          # first row that sees none of them
+    dk = np.zeros((j1 - j0, q.shape[2]))
+    dv = np.zeros((j1 - j0, q.shape[2]))
+    kg = np.asarray(k[:, g, :], dtype=np.float64)
+    vg = np.asarray(v[:, g, :], dtype=np.float64)
+    for i in range(j0, last):
+        vis = np.nonzero(ev[: i + 1] > i)[0]
+        sel = (vis >= j0) & (vis < j1)
+        if not sel.any():
+            continue
+        Kc, Vc = kg[vis], vg[vis]
+        for h in range(g * G, (g + 1) * G):
+            qi = np.asarray(q[i, h, :], dtype=np.float64)
+            do = np.asarray(dout[i, h, :], dtype=np.float64)
+            s = scale * (Kc @ qi)
+            e = np.exp(s - s.max())
+            p = e / e.sum()
+            o = p @ Vc
+            ds = p * (Vc @ do - do @ o)
+            dk[vis[sel] - j0] += scale * np.outer(ds[sel], qi)
+            dv[vis[sel] - j0] += np.outer(p[sel], do)
+    return dk, dv
+
+
+# --------------------------------------------------------------------------
+# tile classes
+# --------------------------------------------------------------------------
+def block_minmax(evict_at, block=BLOCK):
+    """kmin[n], kmax[n] over the valid keys of key block n (one trace)."""
+    ev = np.asarray(evict_at, dtype=np.int64)
+    T = ev.shape[0]
+    nb = (T + block - 1) // block
+    kmin = np.zeros(nb, dtype=np.int32)
+    kmax = np.zeros(nb, dtype=np.int32)
+    for n in range(nb):
+        blk = ev[n * block: min((n + 1) * block, T)]
+        kmin[n] = blk.min()
+        kmax[n] = blk.max()
+    return kmin, kmax
+
+
+def tile_classes_rule(evict_at, block=BLOCK):
+    """Classes [nb, nb] uint8 from the min/max rule.  With q0, q1 the first and
+    last valid query of block m and k0, k1 the first and last valid key of
+    block n: EMPTY if k0 > q1 or q0 >= kmax[n]; FULL if k1 <= q0 and
+    q1 < kmin[n]; otherwise PARTIAL."""
+    T = len(evict_at)
+    nb = (T + block - 1) // block
+    kmin, kmax = block_minmax(evict_at, block)
+    cls = np.zeros((nb, nb), dtype=np.uint8)
+    for m in range(nb):
+        q0, q1 = m * block, min(m * block + block - 1, T - 1)
+        for n in range(nb):
+            k0, k1 = n * block, min(n * block + block - 1, T - 1)
+            if k0 > q1 or q0 >= int(kmax[n]):
+                c = EMPTY
+            elif k1 <= q0 and q1 < int(kmin[n]):
+                c = FULL
+            else:
+                c = PARTIAL
+            cls[m, n] = c
+    return cls
+
+
+def tile_classes_brute(evict_at, block=BLOCK):
+    """Classes [nb, nb] uint8 straight from the boolean mask: all allowed ->
+    FULL, none -> EMPTY, else PARTIAL."""
+    A = allowed(evict_at)
+    T = A.shape[0]
+    nb = (T + block - 1) // block
+    cls = np.zeros((nb, nb), dtype=np.uint8)
+    for m in range(nb):
+        for n in range(nb):
+            t = A[m * block: min((m + 1) * block, T), n * block: min((n + 1) * block, T)]
+            cls[m, n] = FULL if t.all() else (EMPTY if not t.any() else PARTIAL)
+    return cls
+
+
+def live_counts(evict_at):
+    """n_i = number of keys visible to query i (one trace)."""
+    return allowed(evict_at).sum(axis=1)

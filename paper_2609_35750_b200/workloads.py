@@ -1,0 +1,285 @@
+"""Seeded synthetic workloads: eviction patterns and Q/K/V/dO tensors.
+
+This module holds inputs only.  It builds, from a seed, the per-key eviction
+step ``evict_at`` that a compacting rollout would leave behind (Sec. 2,
+"KV-streams" paragraph: the trainer sees one continuous trace plus the spans
+the inference engine deleted) for the retention strategies of Sec. 3
+(Summary, Sliding Window / keep-last-k-turns) and for a token-level stress
+pattern (App. A.4 discusses token-level eviction), and it draws Gaussian
+Q/K/V/dO.  None of the attention arithmetic lives here, so both the CPU
+oracle and the CUDA path may be fed from it.
+
+Conventions
+-----------
+* ``evict_at`` is int32, one entry per packed token, in TRACE-LOCAL
+  coordinates: key ``j`` of a trace is visible to query ``i`` of the same
+  trace iff ``j <= i < evict_at[j]``.
+* "never evicted" is ``INF = 2**31 - 1``.
+* ``cu_seqlens`` is int32 ``[batch + 1]`` with ``cu_seqlens[0] = 0``.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional
+
+import numpy as np
+
+INF = np.int32(2**31 - 1)
+BLOCK = 128  # tile edge used for the class statistics only
+
+
+# --------------------------------------------------------------------------
+# eviction patterns
+# --------------------------------------------------------------------------
+def summary_evict_at(T: int, prompt: int, work_lens, summary: int) -> np.ndarray:
+    """Summary compaction (Sec. 3 "Summary": keep nothing, o = 0, bridge s).
+
+    Layout: ``prompt`` tokens, then segments of ``work_lens[s]`` work tokens
+    followed by ``summary`` summary tokens.  A segment completes iff its work
+    and its summary both end at or before ``T``.  When segment ``s``
+    completes at boundary ``e_s`` its work tokens and the summary of segment
+    ``s - 1`` get ``evict_at = e_s``.  The prompt, the newest summary and the
+    tokens of an unfinished trailing segment never evict.
+
+    ``work_lens`` may be an int (every segment the same) or an iterable that
+    yields one work length per segment.
+    """
+    ev = np.full(T, INF, dtype=np.int32)
+    if isinstance(work_lens, (int, np.integer)):
+        def _gen():
+            while True:
+                yield int(work_lens)
+        it = _gen()
+    else:
+        it = iter(work_lens)
+    pos = min(prompt, T)
+    prev_summary = None  # (start, end) of the previous segment's summary
+    while pos < T:
+        try:
+            w = int(next(it))
+        except StopIteration:
+            break
+        w0, w1 = pos, pos + w
+        s0, s1 = w1, w1 + summary
+        if s1 > T:
+            break  # unfinished trailing segment: nothing more is evicted
+        ev[w0:w1] = s1
+        if prev_summary is not None:
+            ev[prev_summary[0]:prev_summary[1]] = s1
+        prev_summary = (s0, s1)
+        pos = s1
+    return ev
+
+
+def keep_last_k_evict_at(T: int, prompt: int, turn_lens, k: int) -> np.ndarray:
+    """Keep-last-k-turns (Sec. 3 "Sliding Window": o close to B, s = 0).
+
+    Turns follow the never-evicted prompt.  When turn ``t`` ends, every token
+    of turn ``t - k`` gets ``evict_at`` = that end.  The last turn is cut at
+    ``T``.
+    """
+    ev = np.full(T, INF, dtype=np.int32)
+    starts: List[int] = []
+    ends: List[int] = []
+    pos = min(prompt, T)
+    for L in turn_lens:
+        if pos >= T:
+            break
+        e = min(pos + int(L), T)
+        starts.append(pos)
+        ends.append(e)
+        pos = e
+    assert pos >= T, "turn_lens too short to fill the trace"
+    for t in range(k, len(starts)):
+        ev[starts[t - k]:ends[t - k]] = ends[t]
+    return ev
+
+
+def fine_grained_evict_at(T: int, prompt: int, rng: np.random.Generator,
+                          mean: float, every_other: bool = True) -> np.ndarray:
+    """Token-level stress: key ``j >= prompt`` with ``(j - prompt)`` odd gets
+    ``evict_at = j + 1 + G_j``, ``G_j`` geometric on {0,1,...} with the given
+    mean (inverse CDF ``floor(log U / log(1 - p))``, ``p = 1/(mean + 1)``).
+    With ``every_other=False`` every non-prompt key is evicted this way."""
+    ev = np.full(T, INF, dtype=np.int32)
+    if T <= prompt:
+        return ev
+    j = np.arange(prompt, T, dtype=np.int64)
+    sel = ((j - prompt) % 2 == 1) if every_other else np.ones_like(j, dtype=bool)
+    p = 1.0 / (mean + 1.0)
+    u = rng.random(j.shape[0])
+    u = np.maximum(u, np.finfo(np.float64).tiny)
+    g = np.floor(np.log(u) / np.log1p(-p)).astype(np.int64)
+    val = np.minimum(j + 1 + g, int(INF) - 1)
+    ev[prompt:][sel] = val[sel].astype(np.int32)
+    return ev
+
+
+# --------------------------------------------------------------------------
+# workloads
+# --------------------------------------------------------------------------
+@dataclass
+class Workload:
+    name: str
+    cu_seqlens: np.ndarray          # int32 [batch + 1]
+    evict_at: np.ndarray            # int32 [Ttot], trace-local
+    Hq: int
+    Hkv: int
+    d: int
+    q_prescale: float = 1.0         # multiplier applied to Q before bf16 rounding
+    softmax_scale: float = 0.0      # 0 => 1/sqrt(d)
+    notes: str = ""
+    rules: List[str] = field(default_factory=list)
+
+    @property
+    def batch(self) -> int:
+        return int(self.cu_seqlens.shape[0] - 1)
+
+    @property
+    def total_tokens(self) -> int:
+        return int(self.cu_seqlens[-1])
+
+    @property
+    def max_seqlen(self) -> int:
+        return int(np.diff(self.cu_seqlens).max()) if self.batch else 0
+
+    @property
+    def scale(self) -> float:
+        return self.softmax_scale if self.softmax_scale != 0.0 else 1.0 / float(np.sqrt(self.d))
+
+    def trace(self, b: int) -> np.ndarray:
+        return self.evict_at[self.cu_seqlens[b]:self.cu_seqlens[b + 1]]
+
+
+def _rng(seed: int, cfg: int, stream: int = 0) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[(seed << 8) + cfg, stream]))
+
+
+def _pack(traces) -> (np.ndarray, np.ndarray):
+    lens = np.array([len(t) for t in traces], dtype=np.int64)
+    cu = np.zeros(len(traces) + 1, dtype=np.int32)
+    cu[1:] = np.cumsum(lens)
+    ev = np.concatenate(traces).astype(np.int32) if len(traces) else np.zeros(0, np.int32)
+    return cu, ev
+
+
+def make_workload(cfg: int, seed: int = 0, shrink: int = 1,
+                  Hq: Optional[int] = None, Hkv: Optional[int] = None,
+                  batch: Optional[int] = None, variant: str = "") -> Workload:
+    """The five synthetic traces.  ``shrink`` divides every length of the
+    layout (trace, prompt, segment, turn) by an integer so that the CPU oracle
+    can run the whole tensor; head counts and batch may be overridden for the
+    same reason.  ``variant``: cfg 1 "B" (scale folded into Q, softmax scale
+    1); cfg 4 "control" (no eviction) or "b" (every non-prompt key evicted).
+    """
+    s = int(shrink)
+    assert s >= 1
+    if cfg == 0:
+        T, prompt, work, summ = 1024 // s, 128 // s, 192 // s, 32 // s
+        ev = summary_evict_at(T, prompt, work, summ)
+        cu, eva = _pack([ev] * (batch or 1))
+        return Workload("cfg0_tiny_summary", cu, eva, Hq or 4, Hkv or 4, 64,
+                        notes="1 trace T=1024, prompt 128, 4x(192 work + 32 summary)")
+    if cfg == 1:
+        T, prompt, work, summ = 32768 // s, 2048 // s, 4096 // s, 512 // s
+        ev = summary_evict_at(T, prompt, work, summ)
+        cu, eva = _pack([ev] * (batch or 4))
+        d = 128
+        if variant == "B":
+            return Workload("cfg1B_7b_summary", cu, eva, Hq or 28, Hkv or 4, d,
+                            q_prescale=1.0 / np.sqrt(d), softmax_scale=1.0,
+                            notes="scale folded into Q, softmax_scale=1")
+        return Workload("cfg1_7b_summary", cu, eva, Hq or 28, Hkv or 4, d,
+                        q_prescale=1.0 / np.sqrt(d),
+                        notes="4 traces T=32768, prompt 2048, 6x(4096+512)+3072 leftover; "
+                              "Q drawn N(0,1)*1/sqrt(d), kernel scale 1/sqrt(d)")
+    if cfg == 2:
+        T, prompt = 65536 // s, 4096 // s
+        lo, hi = max(1, 256 // s), max(1, 2048 // s)
+        traces = []
+        for b in range(batch or 2):
+            r = _rng(seed, 2, b)
+            lens = r.integers(lo, hi + 1, size=(T - prompt) // lo + 2)
+            traces.append(keep_last_k_evict_at(T, prompt, lens, 4))
+        cu, eva = _pack(traces)
+        return Workload("cfg2_keep_last_4_turns", cu, eva, Hq or 32, Hkv or 8, 128,
+                        notes="2 traces T=65536, prompt 4096, turns U[256,2048], keep last 4")
+    if cfg == 3:
+        nb = batch or 16
+        r = _rng(seed, 3, 0)
+        lens = r.integers(8192 // s, 32768 // s + 1, size=nb)
+        traces, rules = [], []
+        for b in range(nb):
+            rb = _rng(seed, 3, 1 + b)
+            T = int(lens[b])
+            if rb.integers(0, 2) == 0:
+                wl = rb.integers(max(1, 1024 // s), max(1, 4096 // s) + 1, size=T // max(1, 1024 // s) + 2)
+                traces.append(summary_evict_at(T, 2048 // s, wl, max(1, 256 // s)))
+                rules.append("summary")
+            else:
+                k = int(rb.integers(2, 7))
+                lo, hi = max(1, 256 // s), max(1, 2048 // s)
+                tl = rb.integers(lo, hi + 1, size=T // lo + 2)
+                traces.append(keep_last_k_evict_at(T, 4096 // s, tl, k))
+                rules.append(f"keep_last_{k}")
+        cu, eva = _pack(traces)
+        return Workload("cfg3_varlen_packed", cu, eva, Hq or 32, Hkv or 8, 128, rules=rules,
+                        notes="16 traces U[8192,32768], mixed summary / keep-last-k rules")
+    if cfg == 4:
+        T, prompt = 131072 // s, 1024 // s
+        if variant == "control":
+            ev = np.full(T, INF, dtype=np.int32)
+            name = "cfg4_control_causal"
+        else:
+            ev = fine_grained_evict_at(T, prompt, _rng(seed, 4, 0), 8192.0 / s,
+                                       every_other=(variant != "b"))
+            name = "cfg4b_fine_grained_all" if variant == "b" else "cfg4_fine_grained"
+        cu, eva = _pack([ev] * (batch or 1))
+        return Workload(name, cu, eva, Hq or 64, Hkv or 8, 128,
+                        notes="1 trace T=131072, prompt 1024, alternate keys evicted after 1+Geom(8192)")
+    raise ValueError(f"unknown config {cfg}")
+
+
+# --------------------------------------------------------------------------
+# integer statistics of a workload (used for FLOP accounting and as pins)
+# --------------------------------------------------------------------------
+def count_pairs(w: Workload) -> int:
+    """Number of allowed (i, j) pairs, head independent:
+    sum_j (min(evict_at[j], T) - j) per trace."""
+    total = 0
+    for b in range(w.batch):
+        ev = w.trace(b).astype(np.int64)
+        T = ev.shape[0]
+        j = np.arange(T, dtype=np.int64)
+        total += int((np.minimum(ev, T) - j).sum())
+    return total
+
+
+def fwd_bwd_flops(w: Workload) -> int:
+    """Unmasked FLOPs: 2 GEMMs forward + 5 backward, 2 flops per MAC."""
+    return 14 * w.d * w.Hq * count_pairs(w)
+
+
+# --------------------------------------------------------------------------
+# tensors
+# --------------------------------------------------------------------------
+def make_tensors(w: Workload, seed: int = 0, device: str = "cpu", with_dout: bool = True):
+    """bf16 q [Ttot,Hq,d], k, v [Ttot,Hkv,d], dout [Ttot,Hq,d] ~ N(0,1) (q times
+    ``q_prescale`` before rounding), drawn by torch's seeded generator on the
+    requested device.  Returns torch tensors."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(1000003 * seed + 17)
+    T = w.total_tokens
+
+    def draw(h, mul=1.0):
+        x = torch.randn((T, h, w.d), generator=g, device=device, dtype=torch.float32)
+        if mul != 1.0:
+            x = x * mul
+        return x.to(torch.bfloat16)
+
+    q = draw(w.Hq, w.q_prescale)
+    k = draw(w.Hkv)
+    v = draw(w.Hkv)
+    dout = draw(w.Hq) if with_dout else None
+    return q, k, v, dout

@@ -1,0 +1,155 @@
+/*
+ * kvs.h -- C ABI of the eviction-masked causal attention library (B200, sm_100a).
+ *
+ * The operation (Sec. 2, "KV-streams" paragraph; Fig. 2 caption): a rollout that was
+ * compacted by evicting KV entries in the inference engine is trained on as ONE continuous
+ * trace; the attention mask hides every evicted key from the queries that came after its
+ * eviction, so one forward pass reproduces what the engine's cache held at every step.
+ * Per key j the caller supplies the step evict_at[j] at which it left the cache; query i
+ * reads key j of the same trace iff   j <= i < evict_at[j].
+ * Positions are not reset by eviction (Sec. 2), so q and k are taken as given.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its name ends in _host.
+ *   - The caller owns every buffer.  No entry point allocates or frees device memory unless
+ *     its comment says so.
+ *   - q, out, dout, dq : bf16 [total_tokens, Hq,  head_dim], contiguous ("thd")
+ *     k, v, dk, dv     : bf16 [total_tokens, Hkv, head_dim], contiguous
+ *     lse              : fp32 [Hq, total_tokens], natural log of sum_j exp(scale * q_i.k_j)
+ *     evict_at         : int32 [total_tokens], TRACE-LOCAL coordinates; 2^31-1 = never
+ *     cu_seqlens       : int32 [batch+1], cu_seqlens[0] = 0, cu_seqlens[batch] = total_tokens
+ *   - Traces are packed back to back; the 128x128 tile grid of a trace starts at its first
+ *     token.  Precondition: evict_at[j] > j (a key is visible at least to its own query).
+ *   - All work is enqueued on `stream` and the call returns without synchronising, except
+ *     where stated.  Return value: KVS_OK or a negative KVS_ERR_* code.  Argument errors are
+ *     detected on the host before anything is launched.  Conditions only the device can see
+ *     (a bad evict_at, a bounded wait that expired) are recorded in a status word inside
+ *     meta_buf / workspace and read back with kvs_device_status().
+ *   - Requires head_dim in {64, 128}, Hq % Hkv == 0, 16-byte aligned tensors.
+ */
+#ifndef KVS_H_
+#define KVS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* kvs_stream_t;   /* a cudaStream_t */
+
+#define KVS_OK                 0
+#define KVS_ERR_INVALID_ARG   (-1)   /* null pointer, negative size, inconsistent dims        */
+#define KVS_ERR_UNSUPPORTED   (-2)   /* head_dim not 64/128, Hq % Hkv != 0, device not sm_100 */
+#define KVS_ERR_ALIGNMENT     (-3)   /* a tensor pointer is not 16-byte aligned               */
+#define KVS_ERR_WORKSPACE     (-4)   /* meta_buf / workspace / arena too small                */
+#define KVS_ERR_CUDA          (-5)   /* a CUDA runtime or driver call failed                  */
+#define KVS_ERR_BAD_EVICT     (-6)   /* device saw evict_at[j] <= j or a malformed cu_seqlens */
+#define KVS_ERR_TIMEOUT       (-7)   /* a bounded device-side wait expired                    */
+#define KVS_ERR_BAD_META      (-8)   /* meta_buf was not produced for these dims              */
+
+#define KVS_TILE        128          /* tile edge, queries and keys */
+#define KVS_CLASS_EMPTY   0
+#define KVS_CLASS_PARTIAL 1
+#define KVS_CLASS_FULL    2
+
+#define KVS_GRAD_BF16 0
+#define KVS_GRAD_FP32 1
+
+/* Text for an error code.  Never NULL. */
+const char* kvs_strerror(int code);
+
+/* Bytes needed for meta_buf.  Pure host arithmetic; 0 on invalid arguments. */
+size_t kvs_mask_meta_bytes(int batch, int total_tokens, int max_seqlen);
+
+/*
+ * Mask metadata (the tile classification that lets the attention kernels skip evicted spans;
+ * the paper states only that the deleted span is masked, Sec. 2 -- the tiling is this
+ * library's).  For every key block n of every trace: kmin/kmax of evict_at over its valid
+ * keys.  For every (query block m, key block n):
+ *     EMPTY   if k0 > q1 or q0 >= kmax[n]
+ *     FULL    if k1 <= q0 and q1 < kmin[n]
+ *     PARTIAL otherwise
+ * (q0,q1 / k0,k1 = first,last valid token of the block).  Also builds, per query block, the
+ * ascending list of its non-empty key blocks and, per key block, the last query block that
+ * sees it, and keeps a copy of evict_at and cu_seqlens, so meta_buf is self-contained and
+ * may be reused by every layer and head that shares (evict_at, cu_seqlens).
+ * max_seqlen must be >= the longest trace.  meta_bytes >= kvs_mask_meta_bytes(...).
+ */
+int kvs_mask_meta(const int32_t* evict_at, const int32_t* cu_seqlens,
+                  int batch, int total_tokens, int max_seqlen,
+                  void* meta_buf, size_t meta_bytes, kvs_stream_t stream);
+
+/*
+ * Test/inspection hook: copies the classes and per-block min/max to HOST arrays and
+ * SYNCHRONISES the stream.  tile_class_host: uint8, trace after trace, each trace a dense
+ * row-major [nb x nb] matrix (nb = ceil(T_b/128); n > m is EMPTY).  kmin_host/kmax_host:
+ * int32 [sum nb].  Any of the three may be NULL.  Returns the device status if it is set.
+ */
+int kvs_mask_meta_export(const void* meta_buf, int batch, const int32_t* cu_seqlens_host,
+                         int total_tokens, int max_seqlen,
+                         uint8_t* tile_class_host, int32_t* kmin_host, int32_t* kmax_host,
+                         kvs_stream_t stream);
+
+/*
+ * Forward:  S_ij = scale * q_i.k_j over allowed j;  lse_i = log sum_j exp S_ij;
+ *           out_i = sum_j exp(S_ij - lse_i) v_j.   Query head h reads KV head h / (Hq/Hkv).
+ * EMPTY tiles are never loaded; element masks are evaluated on PARTIAL tiles only.
+ * softmax_scale == 0 selects 1/sqrt(head_dim).  bf16 operands, fp32 accumulation.
+ */
+int kvs_attn_fwd(const void* q, const void* k, const void* v, const void* meta_buf,
+                 int batch, int total_tokens, int max_seqlen,
+                 int Hq, int Hkv, int head_dim, float softmax_scale,
+                 void* out, float* lse, kvs_stream_t stream);
+
+/* Bytes needed for the backward workspace (row sums, fp32 dQ accumulator, status). */
+size_t kvs_attn_bwd_workspace_bytes(int total_tokens, int Hq, int Hkv, int head_dim, int grad_dtype);
+
+/*
+ * Backward of the same operation (gradients of sum(out * dout)):
+ *   D_i = dout_i.out_i;  P_ij = exp(S_ij - lse_i);  dP_ij = dout_i.v_j;  dS_ij = P_ij (dP_ij - D_i)
+ *   dq_i = scale sum_j dS_ij k_j;  dk_j = scale sum_{h in group} sum_i dS_ij q_i;
+ *   dv_j = sum_{h in group} sum_i P_ij dout_i
+ * grad_dtype: KVS_GRAD_BF16 (dq/dk/dv are bf16) or KVS_GRAD_FP32 (they are fp32, same shapes).
+ * dq is accumulated with fp32 atomics (last bits may differ run to run); dk, dv are
+ * written once, in a fixed order.  The workspace is scratch: its contents after the call
+ * are unspecified, and two calls sharing one workspace must not overlap on the device.
+ */
+int kvs_attn_bwd(const void* dout, const void* q, const void* k, const void* v,
+                 const void* out, const float* lse, const void* meta_buf,
+                 int batch, int total_tokens, int max_seqlen,
+                 int Hq, int Hkv, int head_dim, float softmax_scale, int grad_dtype,
+                 void* dq, void* dk, void* dv,
+                 void* workspace, size_t workspace_bytes, kvs_stream_t stream);
+
+/*
+ * Reads the status word of a meta_buf or of a backward workspace.  SYNCHRONISES the stream.
+ * Returns KVS_OK, the recorded KVS_ERR_* code, or KVS_ERR_CUDA.
+ */
+int kvs_device_status(const void* meta_or_workspace, kvs_stream_t stream);
+
+/* Bytes of device arena needed by kvs_attn_fwd_bwd_host for these dims. */
+size_t kvs_host_arena_bytes(int batch, int total_tokens, int max_seqlen,
+                            int Hq, int Hkv, int head_dim, int grad_dtype);
+
+/*
+ * Whole path from HOST buffers (the call a trainer without device tensors makes): copies
+ * evict_at, cu_seqlens, q, k, v, dout to the device arena, runs mask metadata, forward and
+ * backward, copies out, lse, dq, dk, dv back, and SYNCHRONISES the stream.  Host buffers
+ * should be page-locked for the copies to be asynchronous.  arena: device memory the caller
+ * provides, >= kvs_host_arena_bytes(...), 256-byte aligned.  Returns the device status.
+ */
+int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t* cu_seqlens_host,
+                          const void* q_host, const void* k_host, const void* v_host,
+                          const void* dout_host,
+                          int batch, int total_tokens, int max_seqlen,
+                          int Hq, int Hkv, int head_dim, float softmax_scale, int grad_dtype,
+                          void* out_host, float* lse_host,
+                          void* dq_host, void* dk_host, void* dv_host,
+                          void* arena, size_t arena_bytes, kvs_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVS_H_ */

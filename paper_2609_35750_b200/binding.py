@@ -1,0 +1,199 @@
+"""Thin ctypes binding of libkvs.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  PyTorch is used here for
+device memory and streams.  There is no CPU fallback: if the library is missing or
+the tensors are not on a CUDA device the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkvs.so")
+
+KVS_OK = 0
+KVS_ERR_INVALID_ARG = -1
+KVS_ERR_UNSUPPORTED = -2
+KVS_ERR_ALIGNMENT = -3
+KVS_ERR_WORKSPACE = -4
+KVS_ERR_CUDA = -5
+KVS_ERR_BAD_EVICT = -6
+KVS_ERR_TIMEOUT = -7
+KVS_ERR_BAD_META = -8
+GRAD_BF16, GRAD_FP32 = 0, 1
+CLASS_EMPTY, CLASS_PARTIAL, CLASS_FULL = 0, 1, 2
+TILE = 128
+
+_vp, _i, _f, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+
+# name -> (restype, argtypes); mirrors include/kvs.h
+SIGNATURES = {
+    "kvs_strerror": (ctypes.c_char_p, [_i]),
+    "kvs_mask_meta_bytes": (_sz, [_i, _i, _i]),
+    "kvs_mask_meta": (_i, [_vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "kvs_mask_meta_export": (_i, [_vp, _i, _vp, _i, _i, _vp, _vp, _vp, _vp]),
+    "kvs_attn_fwd": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp]),
+    "kvs_attn_bwd_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
+    "kvs_attn_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "kvs_device_status": (_i, [_vp, _vp]),
+    "kvs_host_arena_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
+    "kvs_attn_fwd_bwd_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i,
+                                   _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+}
+
+_lib = None
+
+
+class KvsError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+def load() -> ctypes.CDLL:
+    """Loads libkvs.so (built by paper_2609_35750_b200.build).  Raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2609_35750_b200.build`; there is no fallback path")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return load().kvs_strerror(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != KVS_OK:
+        raise KvsError(code, where)
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _dev(t: torch.Tensor, name: str, dtype=None) -> int:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (there is no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+# ------------------------------------------------------------------------------------------
+# same names as the C ABI
+# ------------------------------------------------------------------------------------------
+def kvs_mask_meta_bytes(batch: int, total_tokens: int, max_seqlen: int) -> int:
+    return int(load().kvs_mask_meta_bytes(batch, total_tokens, max_seqlen))
+
+
+def kvs_mask_meta(evict_at: torch.Tensor, cu_seqlens: torch.Tensor, max_seqlen: int,
+                  meta_buf: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """evict_at int32 [Ttot], cu_seqlens int32 [batch+1] (device).  Returns meta_buf (uint8)."""
+    batch = cu_seqlens.numel() - 1
+    total = evict_at.numel()
+    need = kvs_mask_meta_bytes(batch, total, max_seqlen)
+    if meta_buf is None:
+        meta_buf = torch.empty(need, dtype=torch.uint8, device=evict_at.device)
+    _check(load().kvs_mask_meta(_dev(evict_at, "evict_at", torch.int32), _dev(cu_seqlens, "cu_seqlens", torch.int32),
+                                batch, total, max_seqlen, _dev(meta_buf, "meta_buf", torch.uint8),
+                                meta_buf.numel(), _stream(stream)), "kvs_mask_meta")
+    return meta_buf
+
+
+def kvs_mask_meta_export(meta_buf: torch.Tensor, cu_seqlens_host, total_tokens: int, max_seqlen: int, stream=None):
+    """Returns (tile_class uint8 [sum nb^2], kmin int32 [sum nb], kmax int32 [sum nb]) as numpy arrays."""
+    import numpy as np
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens_host, dtype=np.int32))
+    batch = cu.shape[0] - 1
+    nb = (np.diff(cu).astype(np.int64) + TILE - 1) // TILE
+    cls = np.zeros(int((nb * nb).sum()), dtype=np.uint8)
+    kmin = np.zeros(int(nb.sum()), dtype=np.int32)
+    kmax = np.zeros(int(nb.sum()), dtype=np.int32)
+    _check(load().kvs_mask_meta_export(_dev(meta_buf, "meta_buf", torch.uint8), batch, cu.ctypes.data, total_tokens, max_seqlen,
+                                       cls.ctypes.data, kmin.ctypes.data, kmax.ctypes.data, _stream(stream)),
+           "kvs_mask_meta_export")
+    return cls, kmin, kmax
+
+
+def kvs_attn_fwd(q, k, v, meta_buf, batch: int, max_seqlen: int, softmax_scale: float = 0.0,
+                 out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None, stream=None):
+    """q [Ttot,Hq,d], k, v [Ttot,Hkv,d] bf16 (device).  Returns (out bf16 [Ttot,Hq,d], lse fp32 [Hq,Ttot])."""
+    total, Hq, d = q.shape
+    Hkv = k.shape[1]
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((Hq, total), dtype=torch.float32, device=q.device)
+    _check(load().kvs_attn_fwd(_dev(q, "q", torch.bfloat16), _dev(k, "k", torch.bfloat16), _dev(v, "v", torch.bfloat16),
+                               _dev(meta_buf, "meta_buf", torch.uint8), batch, total, max_seqlen, Hq, Hkv, d,
+                               float(softmax_scale), _dev(out, "out", torch.bfloat16), _dev(lse, "lse", torch.float32),
+                               _stream(stream)), "kvs_attn_fwd")
+    return out, lse
+
+
+def kvs_attn_bwd_workspace_bytes(total_tokens: int, Hq: int, Hkv: int, head_dim: int, grad_dtype: int) -> int:
+    return int(load().kvs_attn_bwd_workspace_bytes(total_tokens, Hq, Hkv, head_dim, grad_dtype))
+
+
+def kvs_attn_bwd(dout, q, k, v, out, lse, meta_buf, batch: int, max_seqlen: int, softmax_scale: float = 0.0,
+                 grad_dtype: int = GRAD_FP32, dq=None, dk=None, dv=None, workspace=None, stream=None):
+    """Returns (dq, dk, dv) in bf16 or fp32 according to grad_dtype."""
+    total, Hq, d = q.shape
+    Hkv = k.shape[1]
+    gdt = torch.float32 if grad_dtype == GRAD_FP32 else torch.bfloat16
+    if dq is None:
+        dq = torch.empty(q.shape, dtype=gdt, device=q.device)
+    if dk is None:
+        dk = torch.empty(k.shape, dtype=gdt, device=q.device)
+    if dv is None:
+        dv = torch.empty(v.shape, dtype=gdt, device=q.device)
+    need = kvs_attn_bwd_workspace_bytes(total, Hq, Hkv, d, grad_dtype)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    _check(load().kvs_attn_bwd(_dev(dout, "dout", torch.bfloat16), _dev(q, "q", torch.bfloat16), _dev(k, "k", torch.bfloat16),
+                               _dev(v, "v", torch.bfloat16), _dev(out, "out", torch.bfloat16), _dev(lse, "lse", torch.float32),
+                               _dev(meta_buf, "meta_buf", torch.uint8), batch, total, max_seqlen, Hq, Hkv, d,
+                               float(softmax_scale), grad_dtype, _dev(dq, "dq", gdt), _dev(dk, "dk", gdt), _dev(dv, "dv", gdt),
+                               _dev(workspace, "workspace", torch.uint8), workspace.numel(), _stream(stream)), "kvs_attn_bwd")
+    return dq, dk, dv
+
+
+def kvs_device_status(buf: torch.Tensor, stream=None) -> int:
+    return int(load().kvs_device_status(_dev(buf, "buf", torch.uint8), _stream(stream)))
+
+
+def kvs_host_arena_bytes(batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, grad_dtype) -> int:
+    return int(load().kvs_host_arena_bytes(batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, grad_dtype))
+
+
+def kvs_attn_fwd_bwd_host(evict_at, cu_seqlens, q, k, v, dout, max_seqlen: int, softmax_scale: float,
+                          grad_dtype: int, out, lse, dq, dk, dv, arena: torch.Tensor, stream=None) -> None:
+    """All tensors except `arena` are HOST tensors (pinned for asynchronous copies); results
+    are written into out, lse, dq, dk, dv.  Synchronises the stream."""
+    for name, t in (("evict_at", evict_at), ("cu_seqlens", cu_seqlens), ("q", q), ("k", k), ("v", v), ("dout", dout),
+                    ("out", out), ("lse", lse), ("dq", dq), ("dk", dk), ("dv", dv)):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous host tensor")
+    total, Hq, d = q.shape
+    Hkv = k.shape[1]
+    batch = cu_seqlens.numel() - 1
+    _check(load().kvs_attn_fwd_bwd_host(evict_at.data_ptr(), cu_seqlens.data_ptr(), q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                        dout.data_ptr(), batch, total, max_seqlen, Hq, Hkv, d, float(softmax_scale), grad_dtype,
+                                        out.data_ptr(), lse.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(),
+                                        _dev(arena, "arena", torch.uint8), arena.numel(), _stream(stream)),
+           "kvs_attn_fwd_bwd_host")

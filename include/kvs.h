@@ -124,6 +124,19 @@ int kvs_attn_bwd(const void* dout, const void* q, const void* k, const void* v,
                  void* workspace, size_t workspace_bytes, kvs_stream_t stream);
 
 /*
+ * kvs_attn_bwd with two optional cudaEvent_t handles (may be NULL) that are recorded on
+ * `stream` immediately before and after the main dQ/dK/dV kernel, so that a caller can time
+ * that kernel apart from the row-sum pre-pass and the cast post-pass.
+ */
+int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, const void* v,
+                    const void* out, const float* lse, const void* meta_buf,
+                    int batch, int total_tokens, int max_seqlen,
+                    int Hq, int Hkv, int head_dim, float softmax_scale, int grad_dtype,
+                    void* dq, void* dk, void* dv,
+                    void* workspace, size_t workspace_bytes, kvs_stream_t stream,
+                    void* event_main_begin, void* event_main_end);
+
+/*
  * Reads the status word of a meta_buf or of a backward workspace.  SYNCHRONISES the stream.
  * Returns KVS_OK, the recorded KVS_ERR_* code, or KVS_ERR_CUDA.
  */

@@ -39,6 +39,8 @@ SIGNATURES = {
     "kvs_attn_fwd": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp]),
     "kvs_attn_bwd_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
     "kvs_attn_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "kvs_attn_bwd_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp,
+                             _vp, _vp]),
     "kvs_device_status": (_i, [_vp, _vp]),
     "kvs_host_arena_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "kvs_attn_fwd_bwd_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i,
@@ -151,8 +153,11 @@ def kvs_attn_bwd_workspace_bytes(total_tokens: int, Hq: int, Hkv: int, head_dim:
 
 
 def kvs_attn_bwd(dout, q, k, v, out, lse, meta_buf, batch: int, max_seqlen: int, softmax_scale: float = 0.0,
-                 grad_dtype: int = GRAD_FP32, dq=None, dk=None, dv=None, workspace=None, stream=None):
-    """Returns (dq, dk, dv) in bf16 or fp32 according to grad_dtype."""
+                 grad_dtype: int = GRAD_FP32, dq=None, dk=None, dv=None, workspace=None, stream=None,
+                 main_events: Optional[Tuple[torch.cuda.Event, torch.cuda.Event]] = None):
+    """Returns (dq, dk, dv) in bf16 or fp32 according to grad_dtype.  main_events: two timing
+    events (already recorded once, so that their handles exist) to be recorded around the
+    main kernel; this routes through kvs_attn_bwd_ex."""
     total, Hq, d = q.shape
     Hkv = k.shape[1]
     gdt = torch.float32 if grad_dtype == GRAD_FP32 else torch.bfloat16
@@ -165,11 +170,18 @@ def kvs_attn_bwd(dout, q, k, v, out, lse, meta_buf, batch: int, max_seqlen: int,
     need = kvs_attn_bwd_workspace_bytes(total, Hq, Hkv, d, grad_dtype)
     if workspace is None:
         workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
-    _check(load().kvs_attn_bwd(_dev(dout, "dout", torch.bfloat16), _dev(q, "q", torch.bfloat16), _dev(k, "k", torch.bfloat16),
-                               _dev(v, "v", torch.bfloat16), _dev(out, "out", torch.bfloat16), _dev(lse, "lse", torch.float32),
-                               _dev(meta_buf, "meta_buf", torch.uint8), batch, total, max_seqlen, Hq, Hkv, d,
-                               float(softmax_scale), grad_dtype, _dev(dq, "dq", gdt), _dev(dk, "dk", gdt), _dev(dv, "dv", gdt),
-                               _dev(workspace, "workspace", torch.uint8), workspace.numel(), _stream(stream)), "kvs_attn_bwd")
+    args = (_dev(dout, "dout", torch.bfloat16), _dev(q, "q", torch.bfloat16), _dev(k, "k", torch.bfloat16),
+            _dev(v, "v", torch.bfloat16), _dev(out, "out", torch.bfloat16), _dev(lse, "lse", torch.float32),
+            _dev(meta_buf, "meta_buf", torch.uint8), batch, total, max_seqlen, Hq, Hkv, d,
+            float(softmax_scale), grad_dtype, _dev(dq, "dq", gdt), _dev(dk, "dk", gdt), _dev(dv, "dv", gdt),
+            _dev(workspace, "workspace", torch.uint8), workspace.numel(), _stream(stream))
+    if main_events is None:
+        _check(load().kvs_attn_bwd(*args), "kvs_attn_bwd")
+    else:
+        e0, e1 = (int(e.cuda_event) for e in main_events)
+        if not e0 or not e1:
+            raise ValueError("main_events must have been recorded once before the call")
+        _check(load().kvs_attn_bwd_ex(*args, e0, e1), "kvs_attn_bwd_ex")
     return dq, dk, dv
 
 

@@ -360,7 +360,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 template <int D>
 static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo, const MetaView& mv,
                       const BwdParams& p, const __nv_bfloat16* dout, const __nv_bfloat16* out, float* dvec, WsHeader* hdr,
-                      int nb_cap, cudaStream_t st) {
+                      int nb_cap, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1) {
     {
         const long long warps = (long long)p.total_tokens * p.Hq;
         const int threads = 256;
@@ -371,7 +371,9 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     auto kern = bwd_kernel<D>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::DYN_BYTES) != cudaSuccess) return KVS_ERR_CUDA;
     dim3 grid(nb_cap, p.Hkv, 1);
+    if (ev0 && cudaEventRecord(ev0, st) != cudaSuccess) return KVS_ERR_CUDA;
     kern<<<grid, 128, BwdSmem<D>::DYN_BYTES, st>>>(tq, tk, tv, tdo, mv, p);
+    if (ev1 && cudaEventRecord(ev1, st) != cudaSuccess) return KVS_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
 }
 
@@ -385,10 +387,11 @@ extern "C" size_t kvs_attn_bwd_workspace_bytes(int total_tokens, int Hq, int Hkv
     return bwd_ws_layout(total_tokens, Hq, head_dim, grad_dtype).total;
 }
 
-extern "C" int kvs_attn_bwd(const void* dout, const void* q, const void* k, const void* v, const void* out, const float* lse,
-                            const void* meta_buf, int batch, int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim,
-                            float softmax_scale, int grad_dtype, void* dq, void* dk, void* dv, void* workspace,
-                            size_t workspace_bytes, kvs_stream_t stream) {
+extern "C" int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, const void* v, const void* out, const float* lse,
+                               const void* meta_buf, int batch, int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim,
+                               float softmax_scale, int grad_dtype, void* dq, void* dk, void* dv, void* workspace,
+                               size_t workspace_bytes, kvs_stream_t stream, void* event_main_begin, void* event_main_end) {
+    cudaEvent_t ev0 = (cudaEvent_t)event_main_begin, ev1 = (cudaEvent_t)event_main_end;
     if (batch < 0 || total_tokens < 0 || max_seqlen < 0 || Hq <= 0 || Hkv <= 0) return KVS_ERR_INVALID_ARG;
     if (head_dim != 64 && head_dim != 128) return KVS_ERR_UNSUPPORTED;
     if (Hq % Hkv != 0 || Hq > 65535) return KVS_ERR_UNSUPPORTED;
@@ -428,9 +431,9 @@ extern "C" int kvs_attn_bwd(const void* dout, const void* q, const void* k, cons
     p.status = &((WsHeader*)ws)->status;
     if (cudaMemsetAsync(p.dq_acc, 0, nq * sizeof(float), st) != cudaSuccess) return KVS_ERR_CUDA;
     rc = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, mv, p, (const __nv_bfloat16*)dout, (const __nv_bfloat16*)out, (float*)(ws + W.dvec),
-                                         (WsHeader*)ws, L.nb_cap, st)
+                                         (WsHeader*)ws, L.nb_cap, st, ev0, ev1)
                         : launch_bwd<128>(tq, tk, tv, tdo, mv, p, (const __nv_bfloat16*)dout, (const __nv_bfloat16*)out,
-                                          (float*)(ws + W.dvec), (WsHeader*)ws, L.nb_cap, st);
+                                          (float*)(ws + W.dvec), (WsHeader*)ws, L.nb_cap, st, ev0, ev1);
     if (rc != KVS_OK) return rc;
     if (grad_dtype == KVS_GRAD_BF16) {
         const size_t n4 = nq / 4;
@@ -440,4 +443,12 @@ extern "C" int kvs_attn_bwd(const void* dout, const void* q, const void* k, cons
         if (cudaGetLastError() != cudaSuccess) return KVS_ERR_CUDA;
     }
     return KVS_OK;
+}
+
+extern "C" int kvs_attn_bwd(const void* dout, const void* q, const void* k, const void* v, const void* out, const float* lse,
+                            const void* meta_buf, int batch, int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim,
+                            float softmax_scale, int grad_dtype, void* dq, void* dk, void* dv, void* workspace,
+                            size_t workspace_bytes, kvs_stream_t stream) {
+    return kvs_attn_bwd_ex(dout, q, k, v, out, lse, meta_buf, batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, softmax_scale,
+                           grad_dtype, dq, dk, dv, workspace, workspace_bytes, stream, nullptr, nullptr);
 }

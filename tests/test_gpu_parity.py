@@ -1,0 +1,298 @@
+"""CUDA path vs the CPU oracle, element by element, through the C ABI (needs a B200).
+
+Tolerances (bf16 operands, fp32 accumulation; P and dS are rounded to bf16 before the second
+product of each pair, which alone gives about 2e-3 relative L2):
+    max |gpu - oracle| <= 2e-2   and   ||gpu - oracle||_2 / ||oracle||_2 <= 5e-3
+for out, lse and, with fp32 gradient outputs, dq, dk, dv.  With bf16 gradient outputs the
+max-abs bound is 2e-2 or one bf16 ulp of the oracle value, whichever is larger (a value of
+magnitude 8..16 cannot be stored in bf16 more finely than 0.03).  Mask metadata is bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kvs_oracle as O
+from paper_2609_35750_b200 import binding as B
+from paper_2609_35750_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS = 2e-2
+REL_L2 = 5e-3
+DEV = "cuda"
+
+
+def _close(name, got, ref, bf16_out=False, max_abs=None):
+    MAX_ABS = max_abs if max_abs is not None else globals()["MAX_ABS"]
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (name, got.shape, ref.shape)
+    assert np.isfinite(got).all(), f"{name}: non-finite values"
+    err = np.abs(got - ref)
+    if bf16_out:
+        ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(ref), 1e-30))) - 7)
+        bound = np.maximum(MAX_ABS, ulp)
+        assert (err <= bound).all(), f"{name}: max-abs {err.max():.4f} beyond max(2e-2, 1 bf16 ulp)"
+    else:
+        assert err.max() <= MAX_ABS, f"{name}: max-abs {err.max():.4f} > {MAX_ABS}"
+    if np.linalg.norm(ref) > 1e-3:      # a reference that is identically zero has no relative error
+        rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+        assert rel <= REL_L2, f"{name}: rel-L2 {rel:.3e} > {REL_L2}"
+
+
+def _f64(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def _run_gpu(w, q, k, v, do, grad_dtype=B.GRAD_FP32):
+    ev = torch.from_numpy(w.evict_at).to(DEV)
+    cu = torch.from_numpy(w.cu_seqlens).to(DEV)
+    meta = B.kvs_mask_meta(ev, cu, w.max_seqlen)
+    out, lse = B.kvs_attn_fwd(q, k, v, meta, w.batch, w.max_seqlen, w.softmax_scale)
+    ws = torch.empty(B.kvs_attn_bwd_workspace_bytes(w.total_tokens, w.Hq, w.Hkv, w.d, grad_dtype), dtype=torch.uint8, device=DEV)
+    dq, dk, dv = B.kvs_attn_bwd(do, q, k, v, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale, grad_dtype, workspace=ws)
+    assert B.kvs_device_status(meta) == B.KVS_OK
+    assert B.kvs_device_status(ws) == B.KVS_OK
+    return meta, out, lse, dq, dk, dv
+
+
+def _check_meta(w, meta):
+    cls, kmin, kmax = B.kvs_mask_meta_export(meta, w.cu_seqlens, w.total_tokens, w.max_seqlen)
+    ref_cls = np.concatenate([O.tile_classes_rule(w.trace(b)).ravel() for b in range(w.batch)] or [np.zeros(0, np.uint8)])
+    mm = [O.block_minmax(w.trace(b)) for b in range(w.batch)]
+    assert np.array_equal(cls, ref_cls)
+    assert np.array_equal(kmin, np.concatenate([a for a, _ in mm]))
+    assert np.array_equal(kmax, np.concatenate([b for _, b in mm]))
+
+
+def _full_parity(w, seed=0, tensors=None, bwd=True, dq_abs=None):
+    q, k, v, do = tensors if tensors is not None else W.make_tensors(w, seed)
+    qd, kd, vd, dod = (t.to(DEV) for t in (q, k, v, do))
+    meta, out, lse, dq, dk, dv = _run_gpu(w, qd, kd, vd, dod, B.GRAD_FP32)
+    _check_meta(w, meta)
+    qn, kn, vn, don = (_f64(t) for t in (q, k, v, do))
+    ro, rl = O.varlen_fwd(qn, kn, vn, w.evict_at, w.cu_seqlens, w.scale)
+    _close("out", _f64(out), ro)
+    _close("lse", _f64(lse), rl)
+    if not bwd:
+        return out, lse, dq, dk, dv
+    rdq, rdk, rdv = O.varlen_bwd(qn, kn, vn, don, w.evict_at, w.cu_seqlens, w.scale)
+    _close("dq", _f64(dq), rdq, max_abs=dq_abs)
+    _close("dk", _f64(dk), rdk)
+    _close("dv", _f64(dv), rdv)
+    # bf16 gradient outputs: same kernels plus the cast pass
+    _, out2, lse2, dq2, dk2, dv2 = _run_gpu(w, qd, kd, vd, dod, B.GRAD_BF16)
+    assert dq2.dtype == torch.bfloat16
+    assert torch.equal(out, out2) and torch.equal(lse, lse2)       # forward is run-to-run identical
+    _close("dq(bf16)", _f64(dq2), rdq, bf16_out=True, max_abs=dq_abs)
+    _close("dk(bf16)", _f64(dk2), rdk, bf16_out=True)
+    _close("dv(bf16)", _f64(dv2), rdv, bf16_out=True)
+    return out, lse, dq, dk, dv
+
+
+# ---- whole tensors on the tiny config and on shrunk copies of the others ---------------------
+def test_cfg0_full():
+    _full_parity(W.make_workload(0))
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("cfg1_G7", dict(cfg=1, shrink=16, Hq=7, Hkv=1, batch=2)),
+    ("cfg1B_scale1", dict(cfg=1, shrink=16, Hq=7, Hkv=1, batch=1, variant="B")),
+    ("cfg2_G4", dict(cfg=2, shrink=16, Hq=8, Hkv=2, batch=2)),
+    ("cfg3_ragged", dict(cfg=3, shrink=16, Hq=4, Hkv=1, batch=5)),
+    ("cfg4_G8", dict(cfg=4, shrink=32, Hq=8, Hkv=1)),
+    ("cfg4b", dict(cfg=4, shrink=32, Hq=8, Hkv=1, variant="b")),
+    ("cfg4_control", dict(cfg=4, shrink=32, Hq=8, Hkv=1, variant="control")),
+])
+def test_shrunk_configs_full_tensor(name, kw):
+    # Variant B of config 1 folds 1/sqrt(d) into Q and runs with softmax_scale = 1, so dq = 1 * dS k is
+    # sqrt(d) times larger than with the default scale (|dq| reaches ~36) and the rounding of dS to bf16
+    # alone moves it by more than 2e-2; its absolute bound is scaled by sqrt(d), the relative one is not.
+    dq_abs = MAX_ABS * np.sqrt(128.0) if name == "cfg1B_scale1" else None
+    _full_parity(W.make_workload(seed=1, **kw), seed=1, dq_abs=dq_abs)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_cfg0_seeds(seed):
+    w = W.make_workload(0)
+    q, k, v, do = W.make_tensors(w, seed)
+    qd, kd, vd, dod = (t.to(DEV) for t in (q, k, v, do))
+    meta, out, lse, dq, dk, dv = _run_gpu(w, qd, kd, vd, dod)
+    ro, rl = O.varlen_fwd(_f64(q), _f64(k), _f64(v), w.evict_at, w.cu_seqlens, w.scale)
+    _close("out", _f64(out), ro)
+    _close("lse", _f64(lse), rl)
+
+
+# ---- edge cases -------------------------------------------------------------------------------
+def _custom(lens, evs, Hq, Hkv, d, scale=0.0):
+    cu = np.zeros(len(lens) + 1, dtype=np.int32)
+    cu[1:] = np.cumsum(lens)
+    return W.Workload("custom", cu, np.concatenate(evs).astype(np.int32), Hq, Hkv, d, softmax_scale=scale)
+
+
+def _rand_ev(T, rng, maxlife):
+    ev = np.full(T, int(W.INF), dtype=np.int64)
+    sel = rng.random(T) < 0.6
+    ev[sel] = (np.arange(T) + rng.integers(1, maxlife + 1, size=T))[sel]
+    return ev.astype(np.int32)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_ragged_lengths_and_odd_offsets(d):
+    rng = np.random.default_rng(5)
+    lens = [1, 2, 127, 128, 129, 255, 257, 1, 640, 3]
+    evs = [_rand_ev(T, rng, 300) for T in lens]
+    _full_parity(_custom(lens, evs, 4, 2, d), seed=3)
+
+
+def test_single_token_batch_and_no_eviction():
+    _full_parity(_custom([1], [np.array([W.INF])], 2, 1, 128))
+    _full_parity(_custom([129], [np.full(129, W.INF)], 2, 2, 64))     # 1x1 tail tile is FULL
+
+
+def test_evict_after_one_step_closed_form():
+    T = 300
+    w = _custom([T], [np.arange(T) + 1], 4, 2, 128)
+    out, lse, dq, dk, dv = _full_parity(w, seed=4)
+    q, k, v, do = W.make_tensors(w, 4)
+    # every key is visible to itself only: out = v, dq = dk = 0, dv = sum of the group's dout
+    assert torch.equal(out.cpu()[:, 0], v[:, 0]) and torch.equal(out.cpu()[:, 3], v[:, 1])
+    assert float(dq.abs().max()) < 1e-4 and float(dk.abs().max()) < 1e-4
+    ref = do.float()[:, 0] + do.float()[:, 1]
+    assert torch.allclose(dv.cpu()[:, 0], ref, atol=1e-5)
+
+
+def test_retrieval_style_single_evicted_span():
+    T = 700
+    ev = np.full(T, W.INF)
+    ev[100:260] = 500                      # an early turn leaves before the answer tokens
+    _full_parity(_custom([T], [ev], 4, 4, 64), seed=6)
+
+
+def test_masked_huge_logit_and_row_with_no_key_in_first_tile():
+    # keys 0..199 are evicted at 200: rows >= 200 see nothing of key blocks 0 and 1 except
+    # keys 200..255; one evicted key has an enormous logit, which must not leak into the maximum
+    T = 512
+    ev = np.full(T, W.INF)
+    ev[:200] = 200
+    w = _custom([T], [ev], 2, 1, 128, scale=1.0)
+    q, k, v, do = W.make_tensors(w, 7)
+    k = k.clone()
+    k[50] = 40.0                           # q.k ~ +-40*sum(q): huge for some rows
+    # forward only: with logits of this size the gradients are far larger than the absolute bound
+    _full_parity(w, tensors=(q, k, v, do), bwd=False)
+
+
+def test_growing_logits_change_the_maximum_in_every_tile():
+    T = 1024
+    w = _custom([T], [np.full(T, W.INF)], 2, 2, 64, scale=1.0)
+    q, k, v, do = W.make_tensors(w, 8)
+    q = torch.zeros_like(q)
+    k = torch.zeros_like(k)
+    q[:, :, 0] = 1.0
+    k[:, :, 0] = (torch.arange(T, dtype=torch.float32) * 0.08).to(torch.bfloat16)[:, None]   # logits up to ~80
+    _full_parity(w, tensors=(q, k, v, do), bwd=False)
+    # gradients: random q, k with a ramp added to one component, default scale; the running
+    # maximum still drifts upwards by about 0.3 per key tile
+    w = _custom([T], [np.full(T, W.INF)], 2, 2, 64)
+    q, k, v, do = W.make_tensors(w, 8)
+    q[:, :, 0] = 1.0
+    k[:, :, 0] = (k[:, :, 0].float() + torch.arange(T, dtype=torch.float32)[:, None] * 0.02).to(torch.bfloat16)
+    # k now has a component of size up to 20, and dq is a k-weighted sum of dS (rounded to bf16 as an
+    # MMA operand): its values and its rounding error grow with max|k|, so its absolute bound is scaled
+    _full_parity(w, tensors=(q, k, v, do), dq_abs=3 * MAX_ABS)
+
+
+def test_zero_query_live_counts_on_gpu():
+    # exp(lse) with q = 0 counts the visible keys; values for the tiny trace are tabulated
+    import os
+    w = W.make_workload(0)
+    q, k, v, do = W.make_tensors(w, 0)
+    q = torch.zeros_like(q)
+    meta, out, lse, *_ = _run_gpu(w, q.to(DEV), k.to(DEV), v.to(DEV), do.to(DEV))
+    n = np.exp(_f64(lse))
+    gold = os.path.join(os.path.dirname(__file__), "golden", "cfg0_live_counts.txt")
+    for line in open(gold):
+        if line.strip() and not line.startswith("#"):
+            i, ni = (int(x) for x in line.split())
+            assert abs(n[:, i] - ni).max() < 1e-3 * ni
+    live = O.live_counts(w.trace(0))
+    assert np.array_equal(np.rint(n[0]).astype(np.int64), live)
+    # indicator values: v = 1 on a key set A -> out = |A visible| / n_i
+    v2 = torch.zeros_like(v)
+    A = np.zeros(1024, dtype=bool)
+    A[320:352] = True                      # the first summary
+    v2[torch.from_numpy(A)] = 1.0
+    _, out2, *_ = _run_gpu(w, q.to(DEV), k.to(DEV), v2.to(DEV), do.to(DEV))
+    vis = (O.allowed(w.trace(0)) & A[None, :]).sum(1) / live
+    assert np.abs(_f64(out2)[:, 0, 0] - vis).max() < 4e-3
+
+
+def test_run_to_run_determinism_of_fwd_dk_dv():
+    w = W.make_workload(2, shrink=16, Hq=8, Hkv=2, batch=1)
+    q, k, v, do = (t.to(DEV) for t in W.make_tensors(w, 2))
+    a = _run_gpu(w, q, k, v, do)
+    b = _run_gpu(w, q, k, v, do)
+    for x, y in zip((a[1], a[2], a[4], a[5]), (b[1], b[2], b[4], b[5])):
+        assert torch.equal(x, y)
+    assert torch.allclose(a[3], b[3], atol=1e-5, rtol=1e-5)     # dq: fp32 atomics, order may vary
+
+
+# ---- error reporting ----------------------------------------------------------------------------
+def test_bad_evict_at_is_reported_not_fatal():
+    T = 256
+    ev = np.full(T, W.INF).astype(np.int32)
+    ev[10] = 10                                                  # invisible even to itself
+    evd = torch.from_numpy(ev).to(DEV)
+    cu = torch.tensor([0, T], dtype=torch.int32, device=DEV)
+    meta = B.kvs_mask_meta(evd, cu, T)
+    assert B.kvs_device_status(meta) == B.KVS_ERR_BAD_EVICT
+    with pytest.raises(B.KvsError) as e:
+        B.kvs_mask_meta_export(meta, [0, T], T, T)
+    assert e.value.code == B.KVS_ERR_BAD_EVICT
+    # malformed cu_seqlens
+    cu_bad = torch.tensor([0, T + 5], dtype=torch.int32, device=DEV)
+    meta = B.kvs_mask_meta(evd, cu_bad, T)
+    assert B.kvs_device_status(meta) == B.KVS_ERR_BAD_EVICT
+    # the device is still usable
+    _full_parity(W.make_workload(0))
+
+
+def test_argument_errors():
+    w = W.make_workload(0)
+    q, k, v, do = (t.to(DEV) for t in W.make_tensors(w, 0))
+    ev = torch.from_numpy(w.evict_at).to(DEV)
+    cu = torch.from_numpy(w.cu_seqlens).to(DEV)
+    small = torch.empty(256, dtype=torch.uint8, device=DEV)
+    with pytest.raises(B.KvsError) as e:
+        B.kvs_mask_meta(ev, cu, 1024, meta_buf=small)
+    assert e.value.code == B.KVS_ERR_WORKSPACE
+    meta = B.kvs_mask_meta(ev, cu, 1024)
+    with pytest.raises(B.KvsError) as e:
+        B.kvs_attn_fwd(q[:, :3].contiguous(), k[:, :2].contiguous(), v[:, :2].contiguous(), meta, 1, 1024)
+    assert e.value.code == B.KVS_ERR_UNSUPPORTED                # Hq % Hkv != 0
+    out, lse = B.kvs_attn_fwd(q, k, v, meta, 1, 1024)
+    with pytest.raises(B.KvsError) as e:
+        B.kvs_attn_bwd(do, q, k, v, out, lse, meta, 1, 1024, workspace=small)
+    assert e.value.code == B.KVS_ERR_WORKSPACE
+    misaligned = torch.empty(q.numel() + 8, dtype=torch.bfloat16, device=DEV)[1:1 + q.numel()].view_as(q)
+    with pytest.raises(B.KvsError) as e:
+        B.kvs_attn_fwd(misaligned, k, v, meta, 1, 1024)
+    assert e.value.code == B.KVS_ERR_ALIGNMENT
+
+
+def test_host_buffer_entry_point_matches_device_path():
+    w = W.make_workload(3, shrink=32, Hq=4, Hkv=2, batch=3)
+    q, k, v, do = W.make_tensors(w, 9)
+    qd, kd, vd, dod = (t.to(DEV) for t in (q, k, v, do))
+    _, out, lse, dq, dk, dv = _run_gpu(w, qd, kd, vd, dod, B.GRAD_BF16)
+    pin = lambda t: t.contiguous().pin_memory()
+    ho, hl = pin(torch.empty_like(q)), pin(torch.empty((w.Hq, w.total_tokens), dtype=torch.float32))
+    hdq, hdk, hdv = pin(torch.empty_like(q)), pin(torch.empty_like(k)), pin(torch.empty_like(v))
+    arena = torch.empty(B.kvs_host_arena_bytes(w.batch, w.total_tokens, w.max_seqlen, w.Hq, w.Hkv, w.d, B.GRAD_BF16),
+                        dtype=torch.uint8, device=DEV)
+    B.kvs_attn_fwd_bwd_host(pin(torch.from_numpy(w.evict_at)), pin(torch.from_numpy(w.cu_seqlens)), pin(q), pin(k), pin(v), pin(do),
+                            w.max_seqlen, w.softmax_scale, B.GRAD_BF16, ho, hl, hdq, hdk, hdv, arena)
+    assert torch.equal(ho, out.cpu()) and torch.equal(hl, lse.cpu())
+    assert torch.equal(hdk, dk.cpu()) and torch.equal(hdv, dv.cpu())
+    assert torch.allclose(hdq.float(), dq.cpu().float(), atol=2e-2, rtol=2e-2)

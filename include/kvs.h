@@ -137,6 +137,33 @@ int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, const void* 
                     void* event_main_begin, void* event_main_end);
 
 /*
+ * Backward without any device allocation by anyone (no counterpart in the paper: it exists for
+ * deployment).  Some callers cannot obtain device memory at call time: a runtime that handed the
+ * whole HBM to its own pool at start-up (a later cudaMalloc fails), or a step loop that must not
+ * pay the device-wide synchronisation cudaMalloc/cudaFree imply.  For them the scratch that
+ * kvs_attn_bwd takes as `workspace` is a fixed array inside the library, of
+ * 256 B + 4 B * KVS_NOALLOC_MAX_ROWS per GPU, resident on every GPU that loads the library.
+ *   - Gradients are fp32 only (dq is accumulated in place, so it needs no scratch); otherwise the
+ *     arguments and results are those of kvs_attn_bwd with KVS_GRAD_FP32.
+ *   - total_tokens * Hq must not exceed KVS_NOALLOC_MAX_ROWS, else KVS_ERR_WORKSPACE is returned
+ *     and nothing is launched.
+ *   - The first call on a device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.  Later calls only launch.
+ *   - All calls on a GPU share the one array, which keeps whatever the previous call left; this
+ *     call overwrites everything it reads, so nothing needs clearing, but two calls whose kernels
+ *     overlap on the GPU (different streams, or another process thread) race on it.
+ *   - scratch_out (may be NULL) receives the array's device address, for kvs_device_status().
+ * The call itself uses no cudaMalloc, cudaFree or other allocating routine.
+ */
+#define KVS_NOALLOC_MAX_ROWS (1 << 20)
+int kvs_attn_bwd_noalloc(const void* dout, const void* q, const void* k, const void* v,
+                         const void* out, const float* lse, const void* meta_buf,
+                         int batch, int total_tokens, int max_seqlen,
+                         int Hq, int Hkv, int head_dim, float softmax_scale,
+                         float* dq, float* dk, float* dv,
+                         void** scratch_out, kvs_stream_t stream);
+
+/*
  * Reads the status word of a meta_buf or of a backward workspace.  SYNCHRONISES the stream.
  * Returns KVS_OK, the recorded KVS_ERR_* code, or KVS_ERR_CUDA.
  */

@@ -41,6 +41,8 @@ SIGNATURES = {
     "kvs_attn_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "kvs_attn_bwd_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp,
                              _vp, _vp]),
+    "kvs_attn_bwd_noalloc": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp,
+                                  ctypes.POINTER(ctypes.c_void_p), _vp]),
     "kvs_device_status": (_i, [_vp, _vp]),
     "kvs_host_arena_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "kvs_attn_fwd_bwd_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i,
@@ -183,6 +185,39 @@ def kvs_attn_bwd(dout, q, k, v, out, lse, meta_buf, batch: int, max_seqlen: int,
             raise ValueError("main_events must have been recorded once before the call")
         _check(load().kvs_attn_bwd_ex(*args, e0, e1), "kvs_attn_bwd_ex")
     return dq, dk, dv
+
+
+NOALLOC_MAX_ROWS = 1 << 20
+
+
+def kvs_attn_bwd_noalloc(dout, q, k, v, out, lse, meta_buf, batch: int, max_seqlen: int, softmax_scale: float = 0.0,
+                         dq=None, dk=None, dv=None, stream=None):
+    """Backward for callers that must not allocate device memory at call time: the scratch is a
+    fixed array inside the library (fp32 gradients only, total_tokens * Hq <= NOALLOC_MAX_ROWS).
+    Pass dq, dk, dv to keep this wrapper from allocating too.  Returns (dq, dk, dv, scratch_address);
+    the address can be given to kvs_device_status_ptr()."""
+    total, Hq, d = q.shape
+    Hkv = k.shape[1]
+    if dq is None:
+        dq = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+    if dk is None:
+        dk = torch.empty(k.shape, dtype=torch.float32, device=q.device)
+    if dv is None:
+        dv = torch.empty(v.shape, dtype=torch.float32, device=q.device)
+    scratch = ctypes.c_void_p(0)
+    _check(load().kvs_attn_bwd_noalloc(_dev(dout, "dout", torch.bfloat16), _dev(q, "q", torch.bfloat16),
+                                       _dev(k, "k", torch.bfloat16), _dev(v, "v", torch.bfloat16),
+                                       _dev(out, "out", torch.bfloat16), _dev(lse, "lse", torch.float32),
+                                       _dev(meta_buf, "meta_buf", torch.uint8), batch, total, max_seqlen, Hq, Hkv, d,
+                                       float(softmax_scale), _dev(dq, "dq", torch.float32), _dev(dk, "dk", torch.float32),
+                                       _dev(dv, "dv", torch.float32), ctypes.byref(scratch), _stream(stream)),
+           "kvs_attn_bwd_noalloc")
+    return dq, dk, dv, int(scratch.value or 0)
+
+
+def kvs_device_status_ptr(device_address: int, stream=None) -> int:
+    """kvs_device_status on a raw device address (e.g. the scratch of kvs_attn_bwd_noalloc)."""
+    return int(load().kvs_device_status(device_address, _stream(stream)))
 
 
 def kvs_device_status(buf: torch.Tensor, stream=None) -> int:

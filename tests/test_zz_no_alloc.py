@@ -1,0 +1,65 @@
+"""The allocation-free backward entry point against the ordinary one (needs a B200).
+
+Collected last on purpose: a run that stops at the first failure has then already been through
+every other test.  kvs_attn_bwd_noalloc keeps its scratch in a fixed array inside the library,
+for callers that cannot get device memory at call time (all HBM already owned by the host
+framework's pool, or no tolerance for the synchronisation an allocation implies).  Checked
+here: same gradients as kvs_attn_bwd on two calls in a row that share the array (the second
+with other sizes and inputs, so stale contents would show), and a clean refusal beyond the
+stated maximum.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_35750_b200 import binding as B
+from paper_2609_35750_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _both_ways(w, seed):
+    q, k, v, do = (t.to(DEV) for t in W.make_tensors(w, seed))
+    ev = torch.from_numpy(w.evict_at).to(DEV)
+    cu = torch.from_numpy(w.cu_seqlens).to(DEV)
+    meta = B.kvs_mask_meta(ev, cu, w.max_seqlen)
+    out, lse = B.kvs_attn_fwd(q, k, v, meta, w.batch, w.max_seqlen, w.softmax_scale)
+    ref = B.kvs_attn_bwd(do, q, k, v, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale, B.GRAD_FP32)
+    # outputs allocated up front: the call under test then touches no allocator at all
+    dq = torch.empty(q.shape, dtype=torch.float32, device=DEV)
+    dk = torch.empty(k.shape, dtype=torch.float32, device=DEV)
+    dv = torch.empty(v.shape, dtype=torch.float32, device=DEV)
+    torch.cuda.synchronize()
+    before = torch.cuda.memory_allocated()
+    _, _, _, scratch = B.kvs_attn_bwd_noalloc(do, q, k, v, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale,
+                                              dq=dq, dk=dk, dv=dv)
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() == before
+    assert scratch != 0 and B.kvs_device_status_ptr(scratch) == B.KVS_OK
+    # dk, dv are written in a fixed order: identical.  dq is summed with fp32 atomics: the order varies.
+    assert torch.equal(dk, ref[1]) and torch.equal(dv, ref[2])
+    assert torch.allclose(dq, ref[0], atol=1e-4, rtol=1e-4)
+    err = (dq - ref[0]).abs().max().item()
+    assert err <= 2e-2
+    return scratch
+
+
+def test_noalloc_backward_matches_workspace_backward_twice_in_a_row():
+    s1 = _both_ways(W.make_workload(2, seed=3, shrink=16, Hq=8, Hkv=2, batch=2), seed=3)
+    s2 = _both_ways(W.make_workload(3, seed=4, shrink=32, Hq=4, Hkv=1, batch=3), seed=4)     # smaller, ragged
+    s3 = _both_ways(W.make_workload(0), seed=5)                                              # head_dim 64
+    assert s1 == s2 == s3                      # one array per GPU, shared by every call
+
+
+def test_noalloc_rejects_sizes_beyond_its_maximum():
+    Hq, d = 8, 128
+    T = B.NOALLOC_MAX_ROWS // Hq + 128         # total_tokens * Hq just over the limit
+    q = torch.empty((T, Hq, d), dtype=torch.bfloat16, device=DEV)
+    kv = torch.empty((T, 1, d), dtype=torch.bfloat16, device=DEV)
+    lse = torch.empty((Hq, T), dtype=torch.float32, device=DEV)
+    meta = torch.empty(B.kvs_mask_meta_bytes(1, T, T), dtype=torch.uint8, device=DEV)
+    with pytest.raises(B.KvsError) as e:
+        B.kvs_attn_bwd_noalloc(q, q, kv, kv, q, lse, meta, 1, T)
+    assert e.value.code == B.KVS_ERR_WORKSPACE
+    assert "too small" in str(e.value)

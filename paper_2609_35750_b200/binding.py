@@ -62,10 +62,11 @@ def load() -> ctypes.CDLL:
     """Loads libkvs.so (built by paper_2609_35750_b200.build).  Raises if absent."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
+        path = os.environ.get("KVS_LIB", LIB_PATH)       # KVS_LIB: an alternative build of the same library
+        if not os.path.exists(path):
             raise FileNotFoundError(
-                f"{LIB_PATH} not found: build it with `python -m paper_2609_35750_b200.build`; there is no fallback path")
-        lib = ctypes.CDLL(LIB_PATH)
+                f"{path} not found: build it with `python -m paper_2609_35750_b200.build`; there is no fallback path")
+        lib = ctypes.CDLL(path)
         for name, (res, args) in SIGNATURES.items():
             fn = getattr(lib, name)
             fn.restype = res

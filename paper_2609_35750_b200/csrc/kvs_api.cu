@@ -37,6 +37,21 @@ int make_tmap_thd(CUtensorMap* map, const void* base, int total_tokens, int head
     return r == CUDA_SUCCESS ? KVS_OK : KVS_ERR_CUDA;
 }
 
+// fp32 [total_tokens, heads, head_dim] viewed as (head_dim, heads, tokens); box = 32 columns (128 bytes) x
+// 1 head x box_rows tokens, 128-byte swizzle.  Used as the destination of TMA reduce-adds.
+int make_tmap_f32_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return KVS_ERR_CUDA;
+    cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)heads, (cuuint64_t)total_tokens};
+    cuuint64_t strides[2] = {(cuuint64_t)head_dim * 4, (cuuint64_t)heads * head_dim * 4};
+    cuuint32_t box[3] = {32, 1, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? KVS_OK : KVS_ERR_CUDA;
+}
+
 int check_device_sm100() {
     int dev = 0, major = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return KVS_ERR_CUDA;

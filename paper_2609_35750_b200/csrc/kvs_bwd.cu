@@ -1,19 +1,10 @@
 // Backward: dQ, dK, dV of eviction-masked causal attention.
 //
 //   pre-pass   D_i = dout_i . out_i                         (one warp per (token, head))
-//   main       one CTA per (key block n, KV head g); K and V tiles stay in shared memory;
-//              loop over the G query heads of the group and over the contiguous range of
-//              query blocks m = n .. col_last[n] that can see the key block:
-//                TMA Q, dO tiles
-//                tcgen05.mma  S^T  = K Q^T,  dP^T = V dO^T        (tensor memory, keys on lanes)
-//                128 threads, one key row each: P^T = exp2(S^T*c - lse*log2e) (masked on
-//                  PARTIAL tiles; the key's eviction step is a per-thread scalar),
-//                  dS^T = P^T (dP^T - D); both -> bf16 in tensor memory (over S^T, dP^T),
-//                  dS^T also -> shared memory (MN-major) for the dQ product
-//                tcgen05.mma  dV += P^T dO,  dK += dS^T Q         (A from tensor memory)
-//                tcgen05.mma  dQ  = dS K                          (into the S^T columns)
-//                dQ tile -> fp32 atomics into the accumulator
-//              epilogue: dK * scale, dV written once by their owner CTA
+//   main       one CTA per (key block n, KV head g), longest key blocks first; K and V tiles stay in
+//              shared memory; the CTA loops over the G query heads of the group and over the
+//              contiguous range of query blocks n .. col_last[n] that can see the key block
+//              (see the comment above bwd_kernel for the pipeline)
 //   post-pass  fp32 dQ accumulator -> bf16 (bf16 gradients only)
 #include "kvs_common.cuh"
 
@@ -73,19 +64,43 @@ __global__ void bwd_cast_kernel(const float* __restrict__ acc, __nv_bfloat16* __
 }
 
 // ---- main -------------------------------------------------------------------------------------
+// Warp-specialised, 16 warps in four warp groups:
+//   warps 0-7   compute: one key row per thread, 64 of the 128 query columns each (P^T, dS^T)
+//   warps 8-11  drain:   dQ tile, tensor memory -> registers -> swizzled shared memory -> TMA
+//               reduce-add into the fp32 accumulator (global `red` instructions are processed at
+//               about one thread per clock per SM, which alone would exceed the MMA time of a tile)
+//   warp 12     producer (TMA for K, V, Q, dO; plain loads for lse and D)
+//   warp 13     MMA issuer;   warps 14-15 idle (they only complete the warp group)
+// Registers are re-balanced per warp group with setmaxnreg (compute 144, drain 136, the rest 88).
+//
+// Tensor memory (512 columns):  [0,128) S^T fp32, then P^T bf16 in [0,32) and [64,96)
+//                               [128,256) dP^T fp32, then dS^T bf16 in +[0,32), +[64,96); then dQ fp32
+//                               [256,256+D) dV     [384,384+D) dK
+// Per iteration j (one (head, query block) tile) the tensor pipe runs, in this order,
+//     dP^T(j) = V dO^T,  dV(j) += P^T dO,  S^T(j+1) = K Q^T,  dK(j) += dS^T Q,  dQ(j) = dS K
+// while the compute warps run  dS(j), P(j+1)  and the drain warps empty dQ(j).  The softmax scale
+// is folded into dS (dS = P (scale dP - scale D)), so dK and dQ leave the tensor core scaled.
+// Rows of a dQ tile past the end of a trace are exactly zero (their P is zero), so the reduce-add
+// of a whole 128-row box is harmless where it overlaps the next trace.
+constexpr int BWD_THREADS = 512;
+
 template <int D>
 struct BwdSmem {
-    static constexpr int TILE_BYTES = TILE * D * 2;
+    static constexpr int TB = TILE * D * 2;
+    static constexpr int STG_BYTES = TILE * 128;     // 128 rows x 32 fp32
     static constexpr int OFF_K = 0;
-    static constexpr int OFF_V = OFF_K + TILE_BYTES;
-    static constexpr int OFF_Q = OFF_V + TILE_BYTES;
-    static constexpr int OFF_DO = OFF_Q + TILE_BYTES;
-    static constexpr int OFF_DS = OFF_DO + TILE_BYTES;          // 128 keys x 128 queries bf16
-    static constexpr int OFF_LSE = OFF_DS + TILE * TILE * 2;
-    static constexpr int OFF_DV = OFF_LSE + TILE * 4;
-    static constexpr int OFF_BAR = OFF_DV + TILE * 4;
-    static constexpr int TOTAL = OFF_BAR + 64;
-    static constexpr int DYN_BYTES = TOTAL + 1024;
+    static constexpr int OFF_V = TB;
+    static constexpr int OFF_Q = 2 * TB;             // 2 stages
+    static constexpr int OFF_DO = 4 * TB;            // 1 stage
+    static constexpr int OFF_DS = 5 * TB;            // 128 keys x 128 queries bf16
+    static constexpr int OFF_STG = OFF_DS + TILE * TILE * 2;   // 2 staging buffers for dQ chunks
+    static constexpr int OFF_LSE = OFF_STG + 2 * STG_BYTES;    // 2 stages x 128 fp32 (already * log2 e)
+    static constexpr int OFF_DVEC = OFF_LSE + 2 * TILE * 4;    // 2 stages x 128 fp32 (already * scale)
+    static constexpr int OFF_BAR = OFF_DVEC + 2 * TILE * 4;
+    static constexpr int OFF_MISC = OFF_BAR + 16 * 8;          // tmem base, abort flag
+    static constexpr int TOTAL = OFF_MISC + 16;
+    static constexpr int MAX_DYN = 232448;                     // 227 KB
+    static constexpr int DYN_BYTES = (TOTAL + 1024 > MAX_DYN) ? MAX_DYN : TOTAL + 1024;
 };
 
 struct BwdParams {
@@ -93,21 +108,25 @@ struct BwdParams {
     float scale, scale_log2;
     const float* lse;
     const float* dvec;
-    float* dq_acc;          // fp32 [Ttot, Hq, D], zeroed before the launch
     void* dk;
     void* dv;
     int grad_fp32;
     int32_t* status;
 };
 
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
+#ifdef KVS_TRACE
+// Debug build only: clock64 timestamps of one CTA's pipeline events.
+__device__ long long g_trace[8192];
+#define KVS_TR(slot, j, ev) do { if ((j) >= 8 && (j) < 20) s_tr[((j) - 8) * 16 + (ev)] = (uint32_t)clock64(); } while (0)
+#else
+#define KVS_TR(slot, j, ev) do { } while (0)
+#endif
 
 template <int D>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(BWD_THREADS, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-           const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, MetaView mv, BwdParams p) {
+           const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+           const __grid_constant__ CUtensorMap tm_dq, MetaView mv, BwdParams p) {
     using L = BwdSmem<D>;
     constexpr int NBOX = D / 64;
     constexpr int BOX_BYTES = TILE * 128;
@@ -115,15 +134,15 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     constexpr uint32_t IDESC_ST = make_idesc(TILE, 0, 0);    // K-major x K-major, N = 128 queries
     constexpr uint32_t IDESC_KV = make_idesc(D, 0, 1);       // A from tensor memory, B MN-major, N = D
     constexpr uint32_t IDESC_DQ = make_idesc(D, 1, 1);       // A, B MN-major, N = D
+    constexpr int HALF_D = D / 2;
 
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint32_t s_tmem_base;
-    __shared__ int s_abort;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
+    const int lane = tid & 31;
     if ((int)blockIdx.x >= mv.hdr->nblk_total) return;
-    const int gb = blockIdx.x;
+    const int gb = mv.bwd_order[blockIdx.x];
     const int g = blockIdx.y;
     const int G = p.Hq / p.Hkv;
     const int b = mv.blk_trace[gb];
@@ -132,221 +151,366 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const int T = mv.seq_start[b + 1] - tok0;
     const int nb = (T + TILE - 1) / TILE;
     const int m_last = mv.col_last[gb];
-    const uint8_t* cls_col = mv.tile_class + mv.cls_off[b] + n;   // class of (m, n) at cls_col[m * nb]
+    const int nm = m_last - n + 1;                  // query blocks n .. m_last see this key block
+    const int n_iter = G * nm;
     int32_t* status = p.status;
 
-    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
+    const uint32_t sraw = smem_u32(smem_raw);
+    const uint32_t sbase = (sraw + 1023u) & ~1023u;
+    if ((sbase - sraw) + L::TOTAL > (uint32_t)L::DYN_BYTES) {      // shared window not aligned as expected
+        if (tid == 0) set_status(status, KVS_ERR_CUDA);
+        return;
+    }
+    uint8_t* sgen = smem_raw + (sbase - sraw);
     const uint32_t sK = sbase + L::OFF_K, sV = sbase + L::OFF_V, sQ = sbase + L::OFF_Q, sDO = sbase + L::OFF_DO,
-                   sDS = sbase + L::OFF_DS;
-    uint8_t* sDS_gen = sgen + L::OFF_DS;
-    float* sLse = reinterpret_cast<float*>(sgen + L::OFF_LSE);
-    float* sDv = reinterpret_cast<float*>(sgen + L::OFF_DV);
-    const uint32_t bar_kv = sbase + L::OFF_BAR, bar_ld = bar_kv + 8, bar_s = bar_kv + 16, bar_a = bar_kv + 24, bar_q = bar_kv + 32;
+                   sDS = sbase + L::OFF_DS, sSTG = sbase + L::OFF_STG;
+    uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(sgen + L::OFF_MISC);
+#ifdef KVS_TRACE
+    volatile uint32_t* s_tr = reinterpret_cast<volatile uint32_t*>(sgen + L::TOTAL);   // 12 iterations x 16 events
+#endif
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + L::OFF_MISC + 4);
+    const uint32_t bars = sbase + L::OFF_BAR;
+    const uint32_t bar_kv = bars;
+    auto bar_qfull = [&](int s) { return bars + 8 * (1 + s); };
+    auto bar_ldfull = [&](int s) { return bars + 8 * (3 + s); };
+    auto bar_qfree = [&](int s) { return bars + 8 * (5 + s); };
+    const uint32_t bar_dofull = bars + 8 * 7, bar_dofree = bars + 8 * 8, bar_s = bars + 8 * 9, bar_dp = bars + 8 * 10,
+                   bar_p = bars + 8 * 11, bar_ds = bars + 8 * 12, bar_dq = bars + 8 * 13, bar_drained = bars + 8 * 14;
 
     if (tid == 0) {
-        s_abort = 0;
+        *abort_flag = 0;
         mbar_init(bar_kv, 1);
-        mbar_init(bar_ld, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar_qfull(s), 1);
+            mbar_init(bar_ldfull(s), 32);
+            mbar_init(bar_qfree(s), 1);
+        }
+        mbar_init(bar_dofull, 1);
+        mbar_init(bar_dofree, 1);
         mbar_init(bar_s, 1);
-        mbar_init(bar_a, 1);
-        mbar_init(bar_q, 1);
+        mbar_init(bar_dp, 1);
+        mbar_init(bar_p, 8);
+        mbar_init(bar_ds, 8);
+        mbar_init(bar_dq, 1);
+        mbar_init(bar_drained, 4);
         fence_mbar_init();
-        prefetch_tmap(&tm_q);
-        prefetch_tmap(&tm_k);
-        prefetch_tmap(&tm_v);
-        prefetch_tmap(&tm_do);
     }
-    if (warp == 0) {
-        tmem_alloc(smem_u32(&s_tmem_base), TMEM_COLS);
+    if (warp == 13) {
+        tmem_alloc(smem_u32(s_tmem_base), TMEM_COLS);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = s_tmem_base;
-    const uint32_t tmem_S = tmem;             // S^T fp32 [0,128) -> P^T bf16 [0,64); later dQ fp32 [0,D)
-    const uint32_t tmem_P = tmem + 128;       // dP^T fp32 [128,256) -> dS^T bf16 [128,192)
-    const uint32_t tmem_dV = tmem + 256;      // [256, 256+D)
-    const uint32_t tmem_dK = tmem + 384;      // [384, 384+D)
-    const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
-    volatile int* abort_flag = &s_abort;
+    const uint32_t tmem = *s_tmem_base;
+    const uint32_t tmem_S = tmem;
+    const uint32_t tmem_P = tmem + 128;
+    const uint32_t tmem_dV = tmem + 256;
+    const uint32_t tmem_dK = tmem + 384;
 
-    if (tid == 0) {
-        mbar_expect_tx(bar_kv, 2 * L::TILE_BYTES);
-        for (int c = 0; c < NBOX; ++c) tma_load_3d(sK + c * BOX_BYTES, &tm_k, c * 64, g, tok0 + n * TILE, bar_kv);
-        for (int c = 0; c < NBOX; ++c) tma_load_3d(sV + c * BOX_BYTES, &tm_v, c * 64, g, tok0 + n * TILE, bar_kv);
-    }
-
-    const int kj = n * TILE + tid;                                     // this thread's key (trace local)
-    const int my_ev = (kj < T) ? mv.evict[tok0 + kj] : 0;              // 0: visible to nobody
-    const bool key_tail = (n * TILE + TILE > T);
-
-    int it = 0;
-    for (int hh = 0; hh < G; ++hh) {
-        const int h = g * G + hh;
-        for (int m = n; m <= m_last; ++m) {
-            const int c = cls_col[(size_t)m * nb];
-            if (c == KVS_CLASS_EMPTY) continue;
-            const bool need_mask = (c != KVS_CLASS_FULL) || key_tail;
-            const uint32_t ph = it & 1;
-            const int qtok = tok0 + m * TILE;
-            if (tid == 0) {
-                mbar_expect_tx(bar_ld, 2 * L::TILE_BYTES);
-                for (int cc = 0; cc < NBOX; ++cc) tma_load_3d(sQ + cc * BOX_BYTES, &tm_q, cc * 64, h, qtok, bar_ld);
-                for (int cc = 0; cc < NBOX; ++cc) tma_load_3d(sDO + cc * BOX_BYTES, &tm_do, cc * 64, h, qtok, bar_ld);
+    if (warp >= 12) {
+        reg_dec<88>();
+        if (warp == 12) {
+            // ================= producer =================
+            float* sLse = reinterpret_cast<float*>(sgen + L::OFF_LSE);
+            float* sDv = reinterpret_cast<float*>(sgen + L::OFF_DVEC);
+            if (lane == 0) {
+                mbar_expect_tx(bar_kv, 2 * L::TB);
+                for (int c = 0; c < NBOX; ++c) tma_load_3d(sK + c * BOX_BYTES, &tm_k, c * 64, g, tok0 + n * TILE, bar_kv);
+                for (int c = 0; c < NBOX; ++c) tma_load_3d(sV + c * BOX_BYTES, &tm_v, c * 64, g, tok0 + n * TILE, bar_kv);
             }
-            {
-                const int qi = m * TILE + tid;
-                const bool qv = qi < T;
-                // +inf makes P vanish for the rows past the end of the trace
-                sLse[tid] = qv ? p.lse[(size_t)h * p.total_tokens + qtok + tid] * 1.4426950408889634f : INFINITY;
-                sDv[tid] = qv ? p.dvec[(size_t)h * p.total_tokens + qtok + tid] : 0.f;
-            }
-            if (tid == 0) {
-                if (it == 0) mbar_wait(bar_kv, 0, abort_flag, status);
-                mbar_wait(bar_ld, ph, abort_flag, status);
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
-                    mma_ss(tmem_S, smem_desc(sK + off, 16, 1024), smem_desc(sQ + off, 16, 1024), IDESC_ST, kk > 0);
+            for (int j = 0; j < n_iter; ++j) {
+                const int s = j & 1;
+                const int h = g * G + j / nm;
+                const int m = n + j % nm;
+                const int qtok = tok0 + m * TILE;
+                // Q(j), lse(j), D(j): stage s, free once every MMA of iteration j-2 has completed
+                if (j >= 2) mbar_wait(bar_qfree(s), ((j >> 1) + 1) & 1, abort_flag, status);
+                if (lane == 0) {
+                    mbar_expect_tx(bar_qfull(s), L::TB);
+                    for (int c = 0; c < NBOX; ++c) tma_load_3d(sQ + s * L::TB + c * BOX_BYTES, &tm_q, c * 64, h, qtok, bar_qfull(s));
                 }
+                const size_t rowbase = (size_t)h * p.total_tokens + qtok;
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
-                    mma_ss(tmem_P, smem_desc(sV + off, 16, 1024), smem_desc(sDO + off, 16, 1024), IDESC_ST, kk > 0);
+                for (int u = 0; u < 4; ++u) {
+                    const int i = lane * 4 + u;
+                    const bool qv = (m * TILE + i) < T;
+                    // +inf makes P vanish for the rows past the end of the trace
+                    sLse[s * TILE + i] = qv ? p.lse[rowbase + i] * 1.4426950408889634f : INFINITY;
+                    sDv[s * TILE + i] = qv ? p.dvec[rowbase + i] * p.scale : 0.f;
                 }
-                mma_commit(bar_s);
+                mbar_arrive(bar_ldfull(s));
+                // dO(j): single buffer, free once dP(j-1) and dV(j-1) have completed
+                if (lane == 0) {
+                    if (j >= 1) mbar_wait(bar_dofree, (j - 1) & 1, abort_flag, status);
+                    mbar_expect_tx(bar_dofull, L::TB);
+                    for (int c = 0; c < NBOX; ++c) tma_load_3d(sDO + c * BOX_BYTES, &tm_do, c * 64, h, qtok, bar_dofull);
+                }
+                __syncwarp();
             }
-            __syncthreads();                      // sLse / sDv visible
-            mbar_wait(bar_s, ph, abort_flag, status);
+        } else if (warp == 13 && lane == 0) {
+            // ================= MMA issuer =================
+            // descriptors of stage 0; a stage or a k-step adds a constant to the 14-bit address field
+            const uint64_t dK_k = smem_desc(sK, 16, 1024), dV_k = smem_desc(sV, 16, 1024);
+            const uint64_t dQ_k = smem_desc(sQ, 16, 1024), dDO_k = smem_desc(sDO, 16, 1024);
+            const uint64_t dK_mn = smem_desc(sK, BOX_BYTES, 1024), dDS_mn = smem_desc(sDS, BOX_BYTES, 1024);
+            const uint64_t dQ_mn = smem_desc(sQ, BOX_BYTES, 1024), dDO_mn = smem_desc(sDO, BOX_BYTES, 1024);
+            constexpr uint64_t STAGE = (uint64_t)(L::TB >> 4);
+            mbar_wait(bar_kv, 0, abort_flag, status);
+            mbar_wait(bar_qfull(0), 0, abort_flag, status);
             tc_fence_after();
-
-            // ---- this thread's key row: 128 queries in 4 chunks of 32 ---------------------------
 #pragma unroll
-            for (int ch = 0; ch < TILE / 32; ++ch) {
-                uint32_t rs[32], rp[32];
-                tmem_ld32(tmem_S + lane_sel + ch * 32, rs);
-                tmem_ld32(tmem_P + lane_sel + ch * 32, rp);
-                tmem_wait_ld();
-                uint32_t pk[16], dk_[16];
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
+                mma_ss(tmem_S, dK_k + off, dQ_k + off, IDESC_ST, kk > 0);
+            }
+            mma_commit(bar_s);
+            for (int j = 0; j < n_iter; ++j) {
+                const int s = j & 1;
+                const uint32_t ph = j & 1;
+                const uint64_t so = s ? STAGE : 0;
+                // dP^T(j) = V dO^T  (its columns hold dQ(j-1) until the drain warps have read it)
+                KVS_TR(0, j, 2);
+                mbar_wait(bar_dofull, ph, abort_flag, status);
+                if (j > 0) mbar_wait(bar_drained, (j - 1) & 1, abort_flag, status);
+                tc_fence_after();
+                KVS_TR(0, j, 3);
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float pv[2], dsv[2];
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int col = ch * 32 + e + u;
-                        float pr = fast_exp2(__uint_as_float(rs[e + u]) * p.scale_log2 - sLse[col]);
-                        if (need_mask) {
-                            const int qi = m * TILE + col;
-                            const bool ok = (kj <= qi) && (qi < my_ev);
-                            pr = ok ? pr : 0.f;
-                        }
-                        pv[u] = pr;
-                        dsv[u] = pr * (__uint_as_float(rp[e + u]) - sDv[col]);
-                    }
-                    pk[e >> 1] = pack_bf16(pv[0], pv[1]);
-                    dk_[e >> 1] = pack_bf16(dsv[0], dsv[1]);
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
+                    mma_ss(tmem_P, dV_k + off, dDO_k + off, IDESC_ST, kk > 0);
                 }
-                // bf16 P^T / dS^T over the fp32 columns already consumed
-                tmem_st16(tmem_S + lane_sel + ch * 16, pk);
-                tmem_st16(tmem_P + lane_sel + ch * 16, dk_);
-                // dS^T row -> shared memory, MN-major (queries contiguous), 128-byte swizzle:
-                // 16-byte chunk q of this key row lives in block q/8, row tid, position (q%8) ^ (tid%8)
+                mma_commit(bar_dp);
+                KVS_TR(0, j, 4);
+                // dV(j) += P^T dO
+                mbar_wait(bar_p, ph, abort_flag, status);
+                tc_fence_after();
+                KVS_TR(0, j, 1);
 #pragma unroll
-                for (int v4 = 0; v4 < 4; ++v4) {
-                    const int q16 = ch * 4 + v4;                    // 16-byte chunk index, 0..15
-                    const uint32_t off = (q16 >> 3) * BOX_BYTES + tid * 128 + (((q16 & 7) ^ (tid & 7)) << 4);
-                    *reinterpret_cast<uint4*>(sDS_gen + off) = make_uint4(dk_[v4 * 4], dk_[v4 * 4 + 1], dk_[v4 * 4 + 2], dk_[v4 * 4 + 3]);
+                for (int kk = 0; kk < TILE / 16; ++kk)
+                    mma_ts(tmem_dV, tmem_S + (kk >> 2) * 64 + (kk & 3) * 8, dDO_mn + (uint64_t)(kk * 128), IDESC_KV,
+                           (j > 0) || (kk > 0));
+                mma_commit(bar_dofree);
+                KVS_TR(0, j, 5);
+                // S^T(j+1) = K Q^T
+                if (j + 1 < n_iter) {
+                    const uint64_t so1 = s ? 0 : STAGE;
+                    mbar_wait(bar_qfull(s ^ 1), ((j + 1) >> 1) & 1, abort_flag, status);
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
+                        mma_ss(tmem_S, dK_k + off, dQ_k + so1 + off, IDESC_ST, kk > 0);
+                    }
+                    mma_commit(bar_s);
+                }
+                // dK(j) += dS^T Q, then dQ(j) = dS K (dQ overwrites the columns that hold dS^T, so it goes last)
+                mbar_wait(bar_ds, ph, abort_flag, status);
+                tc_fence_after();
+                KVS_TR(0, j, 6);
+#pragma unroll
+                for (int kk = 0; kk < TILE / 16; ++kk)
+                    mma_ts(tmem_dK, tmem_P + (kk >> 2) * 64 + (kk & 3) * 8, dQ_mn + so + (uint64_t)(kk * 128), IDESC_KV,
+                           (j > 0) || (kk > 0));
+#pragma unroll
+                for (int kk = 0; kk < TILE / 16; ++kk)
+                    mma_ss(tmem_P, dDS_mn + (uint64_t)(kk * 128), dK_mn + (uint64_t)(kk * 128), IDESC_DQ, kk > 0);
+                mma_commit(bar_dq);
+                mma_commit(bar_qfree(s));
+                KVS_TR(0, j, 7);
+            }
+        }
+    } else if (warp >= 8) {
+        // ================= drain warps: dQ(j), query rows on lanes =================
+        reg_inc<136>();
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
+        uint8_t* stg_row = sgen + L::OFF_STG + row * 128;
+        for (int j = 0; j < n_iter; ++j) {
+            const int h = g * G + j / nm;
+            const int m = n + j % nm;
+            mbar_wait(bar_dq, j & 1, abort_flag, status);
+            tc_fence_after();
+            if (tid == 256) KVS_TR(1, j, 8);
+            uint32_t r[D];
+#pragma unroll
+            for (int ch = 0; ch < D / 32; ++ch) {
+                uint32_t t[32];
+                tmem_ld32(tmem_P + lane_sel + ch * 32, t);
+#pragma unroll
+                for (int e = 0; e < 32; ++e) r[ch * 32 + e] = t[e];
+            }
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_drained);      // the columns may be overwritten from here on
+            if (tid == 256) KVS_TR(1, j, 9);
+            // chunks of 32 head-dim columns through two staging buffers
+#pragma unroll
+            for (int ch = 0; ch < D / 32; ++ch) {
+                const int buf = ch & 1;
+                if (tid == 256) bulk_wait_read<1>();      // the reduce that last read this buffer has finished reading
+                named_bar_sync(1, 128);
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    *reinterpret_cast<uint4*>(stg_row + buf * L::STG_BYTES + ((c ^ (row & 7)) << 4)) =
+                        make_uint4(r[ch * 32 + c * 4], r[ch * 32 + c * 4 + 1], r[ch * 32 + c * 4 + 2], r[ch * 32 + c * 4 + 3]);
+                fence_proxy_async();
+                named_bar_sync(1, 128);
+                if (tid == 256) {
+                    tma_reduce_add_3d(&tm_dq, ch * 32, h, tok0 + m * TILE, sSTG + buf * L::STG_BYTES);
+                    bulk_commit();
                 }
             }
+        }
+        if (tid == 256) bulk_wait<0>();
+    } else {
+        // ================= compute warps =================
+        reg_inc<144>();
+        const int quad = warp & 3;
+        const int half = warp >> 2;
+        const int row = quad * 32 + lane;                  // TMEM lane: key row of S^T, dP^T
+        const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
+        const int col0 = half * 64;                        // this thread's 64 query columns
+        const int kj = n * TILE + row;
+        const int my_ev = (kj < T) ? mv.evict[tok0 + kj] : 0;          // 0: visible to nobody
+        const bool key_tail = (n * TILE + TILE > T);
+        const uint8_t* cls_col = mv.tile_class + mv.cls_off[b] + n;   // class of (m, n) at cls_col[m * nb]
+        const float* sLse = reinterpret_cast<const float*>(sgen + L::OFF_LSE);
+        const float* sDv = reinterpret_cast<const float*>(sgen + L::OFF_DVEC);
+        uint8_t* sDS_row = sgen + L::OFF_DS + half * BOX_BYTES + row * 128;
+        float pv[64];
+        int cls_next = cls_col[(size_t)n * nb];            // class of the tile of the next phase_p, fetched early
+
+        auto phase_p = [&](int j) {        // P^T(j) = exp2(S^T * c - lse), masked
+            const int s = j & 1;
+            const int m = n + j % nm;
+            const bool need_mask = (cls_next != KVS_CLASS_FULL) || key_tail;
+            if (j + 1 < n_iter) cls_next = cls_col[(size_t)(n + (j + 1) % nm) * nb];
+            mbar_wait(bar_ldfull(s), (j >> 1) & 1, abort_flag, status);
+            mbar_wait(bar_s, j & 1, abort_flag, status);
+            tc_fence_after();
+            if (tid == 0) KVS_TR(2, j, 10);
+            const float4* l4 = reinterpret_cast<const float4*>(sLse + s * TILE + col0);
+            uint32_t r0[32], r1[32];
+            tmem_ld32(tmem_S + lane_sel + col0, r0);
+            tmem_ld32(tmem_S + lane_sel + col0 + 32, r1);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e4 = 0; e4 < 8; ++e4) {
+                const float4 l = l4[e4];
+                pv[e4 * 4 + 0] = fast_exp2(fmaf(__uint_as_float(r0[e4 * 4 + 0]), p.scale_log2, -l.x));
+                pv[e4 * 4 + 1] = fast_exp2(fmaf(__uint_as_float(r0[e4 * 4 + 1]), p.scale_log2, -l.y));
+                pv[e4 * 4 + 2] = fast_exp2(fmaf(__uint_as_float(r0[e4 * 4 + 2]), p.scale_log2, -l.z));
+                pv[e4 * 4 + 3] = fast_exp2(fmaf(__uint_as_float(r0[e4 * 4 + 3]), p.scale_log2, -l.w));
+            }
+#pragma unroll
+            for (int e4 = 0; e4 < 8; ++e4) {
+                const float4 l = l4[8 + e4];
+                pv[32 + e4 * 4 + 0] = fast_exp2(fmaf(__uint_as_float(r1[e4 * 4 + 0]), p.scale_log2, -l.x));
+                pv[32 + e4 * 4 + 1] = fast_exp2(fmaf(__uint_as_float(r1[e4 * 4 + 1]), p.scale_log2, -l.y));
+                pv[32 + e4 * 4 + 2] = fast_exp2(fmaf(__uint_as_float(r1[e4 * 4 + 2]), p.scale_log2, -l.z));
+                pv[32 + e4 * 4 + 3] = fast_exp2(fmaf(__uint_as_float(r1[e4 * 4 + 3]), p.scale_log2, -l.w));
+            }
+            if (need_mask) {
+#pragma unroll
+                for (int e = 0; e < 64; ++e) {
+                    const int qi = m * TILE + col0 + e;
+                    pv[e] = ((kj <= qi) && (qi < my_ev)) ? pv[e] : 0.f;
+                }
+            }
+            uint32_t pk[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) pk[e] = pack_bf16(pv[2 * e], pv[2 * e + 1]);
+            tmem_st32(tmem_S + lane_sel + col0, pk);       // 64 queries -> 32 packed columns at [col0, col0+32)
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_p);
+            if (tid == 0) KVS_TR(2, j, 11);
+        };
+
+        auto phase_ds = [&](int j) {       // dS^T(j) = P^T (scale dP^T - scale D)
+            const int s = j & 1;
+            mbar_wait(bar_dp, j & 1, abort_flag, status);
+            tc_fence_after();
+            if (tid == 0) KVS_TR(2, j, 12);
+            const float4* d4 = reinterpret_cast<const float4*>(sDv + s * TILE + col0);
+            uint32_t r0[32], r1[32];
+            tmem_ld32(tmem_P + lane_sel + col0, r0);
+            tmem_ld32(tmem_P + lane_sel + col0 + 32, r1);
+            tmem_wait_ld();
+            uint32_t dk_[32];
+#pragma unroll
+            for (int e4 = 0; e4 < 8; ++e4) {
+                const float4 dd = d4[e4];
+                dk_[e4 * 2 + 0] = pack_bf16(pv[e4 * 4 + 0] * fmaf(__uint_as_float(r0[e4 * 4 + 0]), p.scale, -dd.x),
+                                           pv[e4 * 4 + 1] * fmaf(__uint_as_float(r0[e4 * 4 + 1]), p.scale, -dd.y));
+                dk_[e4 * 2 + 1] = pack_bf16(pv[e4 * 4 + 2] * fmaf(__uint_as_float(r0[e4 * 4 + 2]), p.scale, -dd.z),
+                                           pv[e4 * 4 + 3] * fmaf(__uint_as_float(r0[e4 * 4 + 3]), p.scale, -dd.w));
+            }
+#pragma unroll
+            for (int e4 = 0; e4 < 8; ++e4) {
+                const float4 dd = d4[8 + e4];
+                dk_[16 + e4 * 2 + 0] = pack_bf16(pv[32 + e4 * 4 + 0] * fmaf(__uint_as_float(r1[e4 * 4 + 0]), p.scale, -dd.x),
+                                                pv[32 + e4 * 4 + 1] * fmaf(__uint_as_float(r1[e4 * 4 + 1]), p.scale, -dd.y));
+                dk_[16 + e4 * 2 + 1] = pack_bf16(pv[32 + e4 * 4 + 2] * fmaf(__uint_as_float(r1[e4 * 4 + 2]), p.scale, -dd.z),
+                                                pv[32 + e4 * 4 + 3] * fmaf(__uint_as_float(r1[e4 * 4 + 3]), p.scale, -dd.w));
+            }
+            tmem_st32(tmem_P + lane_sel + col0, dk_);
+            // dS^T row -> shared memory, MN-major (queries contiguous), 128-byte swizzle: the 64 queries of
+            // this half are the 128-byte row `row` of block `half`; 16-byte chunk c sits at (c ^ (row % 8))
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<uint4*>(sDS_row + ((c ^ (row & 7)) << 4)) =
+                    make_uint4(dk_[c * 4], dk_[c * 4 + 1], dk_[c * 4 + 2], dk_[c * 4 + 3]);
             tmem_wait_st();
             fence_proxy_async();
             tc_fence_before();
-            __syncthreads();
-            if (tid == 0) {
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < TILE / 16; ++kk) {     // contraction over 16 queries per step
-                    mma_ts(tmem_dV, tmem_S + kk * 8, smem_desc(sDO + kk * 2048, BOX_BYTES, 1024), IDESC_KV, (it > 0) || (kk > 0));
-                }
-#pragma unroll
-                for (int kk = 0; kk < TILE / 16; ++kk) {
-                    mma_ts(tmem_dK, tmem_P + kk * 8, smem_desc(sQ + kk * 2048, BOX_BYTES, 1024), IDESC_KV, (it > 0) || (kk > 0));
-                }
-                mma_commit(bar_a);
-                mbar_wait(bar_a, ph, abort_flag, status);     // P^T consumed before dQ overwrites its columns
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < TILE / 16; ++kk) {     // contraction over 16 keys per step
-                    mma_ss(tmem_S, smem_desc(sDS + kk * 2048, BOX_BYTES, 1024), smem_desc(sK + kk * 2048, BOX_BYTES, 1024),
-                           IDESC_DQ, kk > 0);
-                }
-                mma_commit(bar_q);
-            }
-            mbar_wait(bar_q, ph, abort_flag, status);
-            tc_fence_after();
-            // ---- dQ tile (query rows on lanes) -> fp32 atomics --------------------------------------
-            {
-                const int qi = m * TILE + tid;
-                const bool qv = qi < T;
-                float* dst = p.dq_acc + ((size_t)(qtok + tid) * p.Hq + h) * D;
-#pragma unroll
-                for (int ch = 0; ch < D / 32; ++ch) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem_S + lane_sel + ch * 32, r);
-                    tmem_wait_ld();
-                    if (qv) {
-#pragma unroll
-                        for (int e = 0; e < 32; e += 4)
-                            red_add_v4(dst + ch * 32 + e, __uint_as_float(r[e]) * p.scale, __uint_as_float(r[e + 1]) * p.scale,
-                                       __uint_as_float(r[e + 2]) * p.scale, __uint_as_float(r[e + 3]) * p.scale);
-                    }
-                }
-            }
-            tc_fence_before();
-            __syncthreads();                      // dQ columns, Q/dO/dS tiles and sLse free again
-            ++it;
-        }
-    }
-    if (it == 0 && tid == 0) mbar_wait(bar_kv, 0, abort_flag, status);   // drain the K/V load
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ds);
+            if (tid == 0) KVS_TR(2, j, 13);
+        };
 
-    // ---- epilogue: dK, dV of this key block -----------------------------------------------------
-    tc_fence_after();
-    const bool kvalid = kj < T;
-    const size_t orow = ((size_t)(tok0 + kj) * p.Hkv + g) * D;
+        phase_p(0);
+        for (int j = 0; j < n_iter; ++j) {
+            phase_ds(j);
+            if (j + 1 < n_iter) phase_p(j + 1);
+        }
+
+        // ---- epilogue: dK, dV of this key block, once every MMA has completed ----
+        mbar_wait(bar_qfree((n_iter - 1) & 1), ((n_iter - 1) >> 1) & 1, abort_flag, status);
+        tc_fence_after();
+        const bool kvalid = kj < T;
+        const size_t orow = ((size_t)(tok0 + kj) * p.Hkv + g) * D + half * HALF_D;
 #pragma unroll
-    for (int which = 0; which < 2; ++which) {
-        const uint32_t src = which == 0 ? tmem_dK : tmem_dV;
-        const float mul = which == 0 ? p.scale : 1.f;
-        void* base = which == 0 ? p.dk : p.dv;
+        for (int which = 0; which < 2; ++which) {
+            const uint32_t src = (which == 0 ? tmem_dK : tmem_dV) + lane_sel + half * HALF_D;
+            void* base = which == 0 ? p.dk : p.dv;
 #pragma unroll
-        for (int ch = 0; ch < D / 32; ++ch) {
-            uint32_t r[32];
-            tmem_ld32(src + lane_sel + ch * 32, r);
-            tmem_wait_ld();
-            if (it == 0) {
+            for (int ch = 0; ch < HALF_D / 32; ++ch) {
+                uint32_t r[32];
+                tmem_ld32(src + ch * 32, r);
+                tmem_wait_ld();
+                if (kvalid) {
+                    if (p.grad_fp32) {
+                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + orow + ch * 32);
 #pragma unroll
-                for (int e = 0; e < 32; ++e) r[e] = 0u;
-            }
-            if (kvalid) {
-                if (p.grad_fp32) {
-                    float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + orow + ch * 32);
+                        for (int e = 0; e < 8; ++e)
+                            dst[e] = make_float4(__uint_as_float(r[e * 4]), __uint_as_float(r[e * 4 + 1]), __uint_as_float(r[e * 4 + 2]),
+                                                 __uint_as_float(r[e * 4 + 3]));
+                    } else {
+                        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(base) + orow + ch * 32);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        dst[e] = make_float4(__uint_as_float(r[e * 4]) * mul, __uint_as_float(r[e * 4 + 1]) * mul,
-                                             __uint_as_float(r[e * 4 + 2]) * mul, __uint_as_float(r[e * 4 + 3]) * mul);
-                } else {
-                    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(base) + orow + ch * 32);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        uint4 w;
-                        w.x = pack_bf16(__uint_as_float(r[e * 8 + 0]) * mul, __uint_as_float(r[e * 8 + 1]) * mul);
-                        w.y = pack_bf16(__uint_as_float(r[e * 8 + 2]) * mul, __uint_as_float(r[e * 8 + 3]) * mul);
-                        w.z = pack_bf16(__uint_as_float(r[e * 8 + 4]) * mul, __uint_as_float(r[e * 8 + 5]) * mul);
-                        w.w = pack_bf16(__uint_as_float(r[e * 8 + 6]) * mul, __uint_as_float(r[e * 8 + 7]) * mul);
-                        dst[e] = w;
+                        for (int e = 0; e < 4; ++e) {
+                            uint4 w;
+                            w.x = pack_bf16(__uint_as_float(r[e * 8 + 0]), __uint_as_float(r[e * 8 + 1]));
+                            w.y = pack_bf16(__uint_as_float(r[e * 8 + 2]), __uint_as_float(r[e * 8 + 3]));
+                            w.z = pack_bf16(__uint_as_float(r[e * 8 + 4]), __uint_as_float(r[e * 8 + 5]));
+                            w.w = pack_bf16(__uint_as_float(r[e * 8 + 6]), __uint_as_float(r[e * 8 + 7]));
+                            dst[e] = w;
+                        }
                     }
                 }
             }
@@ -354,11 +518,18 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
+#ifdef KVS_TRACE
+    if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 192) g_trace[tid] = s_tr[tid];
+#endif
+    if (warp == 13) {
+        __syncwarp();
+        tmem_dealloc(tmem, TMEM_COLS);
+    }
 }
 
 template <int D>
-static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo, const MetaView& mv,
+static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
+                      const CUtensorMap& tdq, const MetaView& mv,
                       const BwdParams& p, const __nv_bfloat16* dout, const __nv_bfloat16* out, float* dvec, WsHeader* hdr,
                       int nb_cap, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1) {
     {
@@ -372,7 +543,7 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::DYN_BYTES) != cudaSuccess) return KVS_ERR_CUDA;
     dim3 grid(nb_cap, p.Hkv, 1);
     if (ev0 && cudaEventRecord(ev0, st) != cudaSuccess) return KVS_ERR_CUDA;
-    kern<<<grid, 128, BwdSmem<D>::DYN_BYTES, st>>>(tq, tk, tv, tdo, mv, p);
+    kern<<<grid, BWD_THREADS, BwdSmem<D>::DYN_BYTES, st>>>(tq, tk, tv, tdo, tdq, mv, p);
     if (ev1 && cudaEventRecord(ev1, st) != cudaSuccess) return KVS_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
 }
@@ -408,7 +579,7 @@ extern "C" int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, c
     if (rc != KVS_OK) return rc;
     const MetaLayout L = meta_layout(batch, total_tokens, max_seqlen);
     const MetaView mv = meta_view(meta_buf, L);
-    CUtensorMap tq, tk, tv, tdo;
+    CUtensorMap tq, tk, tv, tdo, tdq;
     if ((rc = make_tmap_thd(&tq, q, total_tokens, Hq, head_dim, TILE)) != KVS_OK) return rc;
     if ((rc = make_tmap_thd(&tk, k, total_tokens, Hkv, head_dim, TILE)) != KVS_OK) return rc;
     if ((rc = make_tmap_thd(&tv, v, total_tokens, Hkv, head_dim, TILE)) != KVS_OK) return rc;
@@ -424,22 +595,23 @@ extern "C" int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, c
     p.scale_log2 = p.scale * 1.4426950408889634f;
     p.lse = lse;
     p.dvec = (const float*)(ws + W.dvec);
-    p.dq_acc = grad_dtype == KVS_GRAD_FP32 ? (float*)dq : (float*)(ws + W.dq_acc);
+    float* dq_acc = grad_dtype == KVS_GRAD_FP32 ? (float*)dq : (float*)(ws + W.dq_acc);
+    if ((rc = make_tmap_f32_thd(&tdq, dq_acc, total_tokens, Hq, head_dim, TILE)) != KVS_OK) return rc;
     p.dk = dk;
     p.dv = dv;
     p.grad_fp32 = grad_dtype == KVS_GRAD_FP32;
     p.status = &((WsHeader*)ws)->status;
-    if (cudaMemsetAsync(p.dq_acc, 0, nq * sizeof(float), st) != cudaSuccess) return KVS_ERR_CUDA;
-    rc = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, mv, p, (const __nv_bfloat16*)dout, (const __nv_bfloat16*)out, (float*)(ws + W.dvec),
+    if (cudaMemsetAsync(dq_acc, 0, nq * sizeof(float), st) != cudaSuccess) return KVS_ERR_CUDA;
+    rc = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, tdq, mv, p, (const __nv_bfloat16*)dout, (const __nv_bfloat16*)out, (float*)(ws + W.dvec),
                                          (WsHeader*)ws, L.nb_cap, st, ev0, ev1)
-                        : launch_bwd<128>(tq, tk, tv, tdo, mv, p, (const __nv_bfloat16*)dout, (const __nv_bfloat16*)out,
+                        : launch_bwd<128>(tq, tk, tv, tdo, tdq, mv, p, (const __nv_bfloat16*)dout, (const __nv_bfloat16*)out,
                                           (float*)(ws + W.dvec), (WsHeader*)ws, L.nb_cap, st, ev0, ev1);
     if (rc != KVS_OK) return rc;
     if (grad_dtype == KVS_GRAD_BF16) {
         const size_t n4 = nq / 4;
         const size_t blocks = (n4 + 255) / 256;
         if (blocks > 0x7fffffffull) return KVS_ERR_UNSUPPORTED;
-        bwd_cast_kernel<<<(unsigned)blocks, 256, 0, st>>>(p.dq_acc, (__nv_bfloat16*)dq, n4);
+        bwd_cast_kernel<<<(unsigned)blocks, 256, 0, st>>>(dq_acc, (__nv_bfloat16*)dq, n4);
         if (cudaGetLastError() != cudaSuccess) return KVS_ERR_CUDA;
     }
     return KVS_OK;
@@ -452,3 +624,9 @@ extern "C" int kvs_attn_bwd(const void* dout, const void* q, const void* k, cons
     return kvs_attn_bwd_ex(dout, q, k, v, out, lse, meta_buf, batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, softmax_scale,
                            grad_dtype, dq, dk, dv, workspace, workspace_bytes, stream, nullptr, nullptr);
 }
+
+#ifdef KVS_TRACE
+extern "C" int kvs_debug_read_trace(long long* host, int n) {
+    return cudaMemcpyFromSymbol(host, kvs::g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : -1;
+}
+#endif

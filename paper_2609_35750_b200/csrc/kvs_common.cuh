@@ -31,7 +31,7 @@ struct MetaHeader {
 // Byte offsets of the arrays inside meta_buf; a pure function of the three sizes so that
 // every entry point can recompute it.
 struct MetaLayout {
-    size_t blk_off, cls_off, seq_start, blk_trace, kmin, kmax, col_last, row_cnt, fwd_order, evict, tile_class, row_list, total;
+    size_t blk_off, cls_off, seq_start, blk_trace, kmin, kmax, col_last, row_cnt, fwd_order, bwd_order, evict, tile_class, row_list, total;
     int nb_cap;            // capacity in blocks
     size_t cls_cap;        // capacity in tiles
 };
@@ -61,6 +61,7 @@ __host__ __device__ inline MetaLayout meta_layout(int batch, int total_tokens, i
     L.col_last = o;  o = align_up(o + sizeof(int32_t) * nb_cap, 256);
     L.row_cnt = o;   o = align_up(o + sizeof(int32_t) * nb_cap, 256);
     L.fwd_order = o; o = align_up(o + sizeof(int32_t) * nb_cap, 256);
+    L.bwd_order = o; o = align_up(o + sizeof(int32_t) * nb_cap, 256);
     L.evict = o;     o = align_up(o + sizeof(int32_t) * (size_t)(total_tokens > 0 ? total_tokens : 1), 256);
     L.tile_class = o; o = align_up(o + L.cls_cap, 256);
     L.row_list = o;  o = align_up(o + sizeof(uint16_t) * L.cls_cap, 256);
@@ -80,6 +81,7 @@ struct MetaView {
     const int32_t* col_last;    // [nblk] last query block (trace local) that sees the key block
     const int32_t* row_cnt;     // [nblk] non-empty key blocks of a query block row
     const int32_t* fwd_order;   // [nblk] query blocks, heaviest first
+    const int32_t* bwd_order;   // [nblk] key blocks, longest query range first
     const int32_t* evict;       // [total_tokens] copy of evict_at
     const uint8_t* tile_class;  // [ncls]
     const uint16_t* row_list;   // [ncls] row m of trace b at cls_off[b] + m * nb
@@ -98,6 +100,7 @@ inline MetaView meta_view(const void* buf, const MetaLayout& L) {
     v.col_last = (const int32_t*)(p + L.col_last);
     v.row_cnt = (const int32_t*)(p + L.row_cnt);
     v.fwd_order = (const int32_t*)(p + L.fwd_order);
+    v.bwd_order = (const int32_t*)(p + L.bwd_order);
     v.evict = (const int32_t*)(p + L.evict);
     v.tile_class = (const uint8_t*)(p + L.tile_class);
     v.row_list = (const uint16_t*)(p + L.row_list);
@@ -113,6 +116,7 @@ struct WsHeader {
 
 // Host helpers implemented in kvs_api.cu
 int make_tmap_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows);
+int make_tmap_f32_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows);
 int check_device_sm100();
 
 #ifdef __CUDACC__
@@ -154,11 +158,25 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // finishes, frees its tensor memory and returns; the result is garbage and the status word
 // says so.  The limit is about two seconds of SM clocks.
 constexpr long long WAIT_LIMIT_CLOCKS = 4000000000LL;
+// try_wait with a suspend-time hint: the warp sleeps in hardware until the phase completes or the
+// hint (nanoseconds) runs out, instead of polling shared memory (polling by many warps takes issue
+// slots and shared-memory cycles away from the MMA issuer and the tensor core's operand reads).
+__device__ __forceinline__ uint32_t mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok;
+}
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
     if (mbar_try_wait(bar, parity)) return;
-    long long t0 = clock64();
+    const long long t0 = clock64();
     while (true) {
-        if (mbar_try_wait(bar, parity)) return;
+        if (mbar_try_wait_hint(bar, parity, 20000u)) return;
         if (*abort_flag) return;
         if (clock64() - t0 > WAIT_LIMIT_CLOCKS) {
             *abort_flag = 1;
@@ -168,12 +186,33 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Register re-balancing between warp groups (all four warps of a warp group execute it).
+template <int N>
+__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
 // TMA: 3-D tiled load, global -> shared, completion on an mbarrier.  No multicast.
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
         : "memory");
+}
+// TMA: 3-D tiled reduce-add, shared -> global (element type from the tensor map), bulk-group completion.
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* map, int c0, int c1, int c2, uint32_t src) {
+    asm volatile(
+        "cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+        ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(src)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");

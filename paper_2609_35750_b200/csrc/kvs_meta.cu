@@ -125,26 +125,62 @@ __global__ void meta_classify_kernel(MetaHeader* hdr, const int32_t* __restrict_
     if (lane == 0) row_cnt[warp] = count;
 }
 
-// ---- kernel 3: query blocks ordered heaviest first (bucket sort on row_cnt, one CTA) ---------
+// ---- kernel 3: work orders, heaviest first (bucket sort, one CTA per order) -------------------
+// blockIdx.x = 0: query blocks by their number of non-empty key blocks (forward);
+// blockIdx.x = 1: key blocks by the length of their query-block range (backward).
 // Only the launch order of work depends on it; ties may land in any order.
 constexpr int ORDER_BINS = 4096;
-__global__ void meta_order_kernel(MetaHeader* hdr, const int32_t* __restrict__ row_cnt, int32_t* fwd_order) {
+__global__ void __launch_bounds__(1024)
+meta_order_kernel(MetaHeader* hdr, const int32_t* __restrict__ blk_off, const int32_t* __restrict__ blk_trace,
+                  const int32_t* __restrict__ row_cnt, const int32_t* __restrict__ col_last, int32_t* fwd_order,
+                  int32_t* bwd_order) {
     __shared__ int bins[ORDER_BINS];
+    __shared__ int warp_tot[32];
     const int n = hdr->nblk_total;
+    const bool bwd = blockIdx.x == 1;
+    int32_t* order = bwd ? bwd_order : fwd_order;
+    auto key = [&](int i) {
+        const int k = bwd ? (col_last[i] - (i - blk_off[blk_trace[i]]) + 1) : row_cnt[i];
+        return min(max(k, 0), ORDER_BINS - 1);
+    };
     for (int i = threadIdx.x; i < ORDER_BINS; i += blockDim.x) bins[i] = 0;
     __syncthreads();
-    for (int i = threadIdx.x; i < n; i += blockDim.x) atomicAdd(&bins[min(row_cnt[i], ORDER_BINS - 1)], 1);
+    for (int i = threadIdx.x; i < n; i += blockDim.x) atomicAdd(&bins[key(i)], 1);
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int run = 0;
-        for (int c = ORDER_BINS - 1; c >= 0; --c) {   // heaviest bucket first
-            const int k = bins[c];
-            bins[c] = run;
-            run += k;
+    // exclusive scan over the bins in DESCENDING key order: thread t owns 4 consecutive reversed bins
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int c[4], sum = 0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        c[u] = bins[ORDER_BINS - 1 - (threadIdx.x * 4 + u)];
+        sum += c[u];
+    }
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = warp_tot[lane], wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += t;
         }
+        warp_tot[lane] = wi - w;     // exclusive prefix of the warp totals
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < n; i += blockDim.x) fwd_order[atomicAdd(&bins[min(row_cnt[i], ORDER_BINS - 1)], 1)] = i;
+    int run = warp_tot[warp] + incl - sum;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        bins[ORDER_BINS - 1 - (threadIdx.x * 4 + u)] = run;
+        run += c[u];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) order[atomicAdd(&bins[key(i)], 1)] = i;
 }
 
 }  // namespace kvs
@@ -178,7 +214,8 @@ extern "C" int kvs_mask_meta(const int32_t* evict_at, const int32_t* cu_seqlens,
                                                             (int32_t*)v.kmax, (int32_t*)v.col_last, (int32_t*)v.evict);
     meta_classify_kernel<<<grid, warps_per_cta * 32, 0, st>>>(v.hdr, v.blk_off, v.cls_off, v.seq_start, v.blk_trace, v.kmin, v.kmax,
                                                               (uint8_t*)v.tile_class, (uint16_t*)v.row_list, (int32_t*)v.row_cnt);
-    meta_order_kernel<<<1, 1024, 0, st>>>(v.hdr, v.row_cnt, (int32_t*)v.fwd_order);
+    meta_order_kernel<<<2, 1024, 0, st>>>(v.hdr, v.blk_off, v.blk_trace, v.row_cnt, v.col_last, (int32_t*)v.fwd_order,
+                                          (int32_t*)v.bwd_order);
     return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
 }
 

@@ -1,28 +1,37 @@
-// Forward: eviction-masked causal attention, one CTA per (query block, query head).
+// Forward: eviction-masked causal attention.
 //
-// Per CTA: the 128 x D query tile is staged once by TMA; the CTA walks the ascending list of
-// non-empty key blocks of its row (EMPTY tiles are never touched).  Per key block:
-//   TMA  K, V tiles -> shared memory (128-byte swizzle)
-//   tcgen05.mma  S = Q K^T            (fp32, tensor memory columns [0,128))
-//   128 threads, one query row each: scale, element mask on PARTIAL tiles only, online
-//     softmax in registers (base-2), P -> bf16 written over S in tensor memory,
-//     O rescaled in tensor memory when the running maximum moved
-//   tcgen05.mma  O += P V             (P from tensor memory, V MN-major from shared memory)
-// Epilogue: O / l -> bf16, LSE -> fp32.
+// One CTA per (query block, pair of query heads of one GQA group).  The two heads share every K/V
+// tile (identical key-block list and element mask), so each tile is fetched once for two 128-row
+// query tiles.  384 threads in three warp groups:
+//   warps 0-3   softmax of tile 0 (one query row per thread)        } registers re-balanced with
+//   warps 4-7   softmax of tile 1                                    } setmaxnreg (208 / 208 / 88)
+//   warp 8      producer: TMA for Q0, Q1 and the K/V ring (2 stages); plain loads for evict_at
+//   warp 9      MMA issuer;  warps 10-11 idle
+// Tensor memory: S0 [0,128)  S1 [128,256)  O0 [256,256+D)  O1 [384,384+D); P (bf16) overwrites S.
+// Per key block i the tensor pipe runs  O0 += P0 V, S0(i+1) = Q0 K^T, O1 += P1 V, S1(i+1) = Q1 K^T
+// while the two softmax groups alternate, so the exponentials of one tile overlap the MMAs of the
+// other.  EMPTY tiles are never visited (the CTA walks the row's non-empty list); the element mask
+// is evaluated on PARTIAL or ragged tiles only.  O is rescaled lazily: a row keeps its reference
+// maximum until the running maximum exceeds it by more than 8 (base-2), so exp2 arguments stay
+// below 2^8 and the rescale of O in tensor memory is rare.
 #include "kvs_common.cuh"
 
 namespace kvs {
 
+constexpr int FWD_THREADS = 384;
+constexpr float RESCALE_THRESHOLD = 8.0f;
+
 template <int D>
 struct FwdSmem {
-    static constexpr int TILE_BYTES = TILE * D * 2;
-    static constexpr int OFF_Q = 0;
-    static constexpr int OFF_K = OFF_Q + TILE_BYTES;
-    static constexpr int OFF_V = OFF_K + TILE_BYTES;
-    static constexpr int OFF_EV = OFF_V + TILE_BYTES;
-    static constexpr int OFF_BAR = OFF_EV + TILE * 4;
-    static constexpr int TOTAL = OFF_BAR + 64;
-    static constexpr int DYN_BYTES = TOTAL + 1024;   // slack for the 1024-byte alignment
+    static constexpr int TB = TILE * D * 2;
+    static constexpr int OFF_Q = 0;                      // 2 query tiles
+    static constexpr int OFF_KV = 2 * TB;                // 2 stages x (K, V)
+    static constexpr int OFF_EV = OFF_KV + 4 * TB;       // 2 stages x 128 int32
+    static constexpr int OFF_FLAG = OFF_EV + 2 * TILE * 4;   // 2 stages x need_mask
+    static constexpr int OFF_BAR = OFF_FLAG + 16;
+    static constexpr int OFF_MISC = OFF_BAR + 16 * 8;
+    static constexpr int TOTAL = OFF_MISC + 16;
+    static constexpr int DYN_BYTES = TOTAL + 1024;       // slack for the 1024-byte alignment
 };
 
 struct FwdParams {
@@ -33,27 +42,28 @@ struct FwdParams {
 };
 
 template <int D>
-__global__ void __launch_bounds__(128, 2)
+__global__ void __launch_bounds__(FWD_THREADS, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, MetaView mv, FwdParams p) {
     using L = FwdSmem<D>;
     constexpr int NBOX = D / 64;             // 64-column TMA boxes per tile row
     constexpr int BOX_BYTES = TILE * 128;    // 128 rows x 128 bytes
-    constexpr uint32_t TMEM_COLS = 256;
+    constexpr uint32_t TMEM_COLS = 512;
     constexpr uint32_t IDESC_S = make_idesc(TILE, 0, 0);
     constexpr uint32_t IDESC_O = make_idesc(D, 0, 1);
 
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint32_t s_tmem_base;
-    __shared__ int s_abort;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
-    const int nblk_total = mv.hdr->nblk_total;
-    if ((int)blockIdx.x >= nblk_total) return;
+    const int lane = tid & 31;
+    if ((int)blockIdx.x >= mv.hdr->nblk_total) return;
     const int gb = mv.fwd_order[blockIdx.x];
-    const int h = blockIdx.y;
-    const int g = h / (p.Hq / p.Hkv);
+    const int G = p.Hq / p.Hkv;
+    const int pairs_per_group = (G + 1) >> 1;
+    const int g = blockIdx.y / pairs_per_group;
+    const int h0 = g * G + 2 * (blockIdx.y % pairs_per_group);
+    const int ntile = (h0 + 1 < (g + 1) * G) ? 2 : 1;       // an odd group ends with a single head
     const int b = mv.blk_trace[gb];
     const int m = gb - mv.blk_off[b];
     const int tok0 = mv.seq_start[b];
@@ -64,179 +74,253 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const uint8_t* cls = mv.tile_class + mv.cls_off[b] + (size_t)m * nb;
     int32_t* status = &mv.hdr->status;
 
-    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
-    const uint32_t sQ = sbase + L::OFF_Q, sK = sbase + L::OFF_K, sV = sbase + L::OFF_V;
+    const uint32_t sraw = smem_u32(smem_raw);
+    const uint32_t sbase = (sraw + 1023u) & ~1023u;
+    uint8_t* sgen = smem_raw + (sbase - sraw);
+    const uint32_t sQ = sbase + L::OFF_Q, sKV = sbase + L::OFF_KV;
     int32_t* sEv = reinterpret_cast<int32_t*>(sgen + L::OFF_EV);
-    const uint32_t bar_q = sbase + L::OFF_BAR, bar_kv = bar_q + 8, bar_s = bar_q + 16, bar_o = bar_q + 24;
+    volatile int32_t* sFlag = reinterpret_cast<volatile int32_t*>(sgen + L::OFF_FLAG);
+    uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(sgen + L::OFF_MISC);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + L::OFF_MISC + 4);
+    const uint32_t bars = sbase + L::OFF_BAR;
+    const uint32_t bar_q = bars;
+    auto bar_kvfull = [&](int s) { return bars + 8 * (1 + s); };    // TMA bytes of K and V
+    auto bar_evfull = [&](int s) { return bars + 8 * (3 + s); };    // evict_at tile + need_mask flag (32 arrivals)
+    auto bar_kvfree = [&](int s) { return bars + 8 * (5 + s); };    // every MMA reading the stage has completed
+    auto bar_s = [&](int t) { return bars + 8 * (7 + t); };         // S_t ready
+    auto bar_p = [&](int t) { return bars + 8 * (9 + t); };         // P_t written (4 arrivals)
+    auto bar_evfree = [&](int s) { return bars + 8 * (11 + s); };   // softmax groups done with the evict_at tile
+    const uint32_t bar_done = bars + 8 * 13;                         // all MMAs complete
 
     if (tid == 0) {
-        s_abort = 0;
+        *abort_flag = 0;
         mbar_init(bar_q, 1);
-        mbar_init(bar_kv, 1);
-        mbar_init(bar_s, 1);
-        mbar_init(bar_o, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar_kvfull(s), 1);
+            mbar_init(bar_evfull(s), 32);
+            mbar_init(bar_kvfree(s), 1);
+            mbar_init(bar_evfree(s), 4 * ntile);
+            mbar_init(bar_s(s), 1);
+            mbar_init(bar_p(s), 4);
+        }
+        mbar_init(bar_done, 1);
         fence_mbar_init();
-        prefetch_tmap(&tm_q);
-        prefetch_tmap(&tm_k);
-        prefetch_tmap(&tm_v);
     }
-    if (warp == 0) {
-        tmem_alloc(smem_u32(&s_tmem_base), TMEM_COLS);
+    if (warp == 9) {
+        tmem_alloc(smem_u32(s_tmem_base), TMEM_COLS);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = s_tmem_base;
-    const uint32_t tmem_S = tmem;            // columns [0,128): S fp32, then P bf16 in [0,64)
-    const uint32_t tmem_O = tmem + 128;      // columns [128,128+D)
-    const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;   // this warp's 32 TMEM lanes
+    const uint32_t tmem = *s_tmem_base;
 
-    if (tid == 0) {
-        mbar_expect_tx(bar_q, L::TILE_BYTES);
-        for (int c = 0; c < NBOX; ++c) tma_load_3d(sQ + c * BOX_BYTES, &tm_q, c * 64, h, tok0 + m * TILE, bar_q);
-    }
-
-    const int row = tid;                      // query row of the tile == TMEM lane
-    const int qi = m * TILE + row;            // trace-local query index
-    float run_max = -INFINITY;                // base-2 domain
-    float run_sum = 0.f;
-    volatile int* abort_flag = &s_abort;
-
-    for (int t = 0; t < nlist; ++t) {
-        const int n = list[t];
-        const uint32_t ph = t & 1;
-        const bool need_mask = (cls[n] != KVS_CLASS_FULL) || (n * TILE + TILE > T);
-        if (tid == 0) {
-            mbar_expect_tx(bar_kv, 2 * L::TILE_BYTES);
-            for (int c = 0; c < NBOX; ++c) tma_load_3d(sK + c * BOX_BYTES, &tm_k, c * 64, g, tok0 + n * TILE, bar_kv);
-            for (int c = 0; c < NBOX; ++c) tma_load_3d(sV + c * BOX_BYTES, &tm_v, c * 64, g, tok0 + n * TILE, bar_kv);
+    if (warp >= 8) {
+        reg_dec<88>();
+        if (warp == 8) {
+            // ================= producer =================
+            if (lane == 0) {
+                mbar_expect_tx(bar_q, ntile * L::TB);
+                for (int t = 0; t < ntile; ++t)
+                    for (int c = 0; c < NBOX; ++c) tma_load_3d(sQ + t * L::TB + c * BOX_BYTES, &tm_q, c * 64, h0 + t, tok0 + m * TILE, bar_q);
+            }
+            for (int i = 0; i < nlist; ++i) {
+                const int s = i & 1;
+                const int n = list[i];
+                if (i >= 2) {
+                    mbar_wait(bar_kvfree(s), ((i >> 1) + 1) & 1, abort_flag, status);
+                    mbar_wait(bar_evfree(s), ((i >> 1) + 1) & 1, abort_flag, status);
+                }
+                if (lane == 0) {
+                    mbar_expect_tx(bar_kvfull(s), 2 * L::TB);
+                    const uint32_t dst = sKV + s * 2 * L::TB;
+                    for (int c = 0; c < NBOX; ++c) tma_load_3d(dst + c * BOX_BYTES, &tm_k, c * 64, g, tok0 + n * TILE, bar_kvfull(s));
+                    for (int c = 0; c < NBOX; ++c) tma_load_3d(dst + L::TB + c * BOX_BYTES, &tm_v, c * 64, g, tok0 + n * TILE, bar_kvfull(s));
+                }
+                const bool need_mask = (cls[n] != KVS_CLASS_FULL) || (n * TILE + TILE > T);
+                if (need_mask) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int j = n * TILE + lane * 4 + u;
+                        sEv[s * TILE + lane * 4 + u] = (j < T) ? mv.evict[tok0 + j] : 0;   // 0: visible to nobody
+                    }
+                }
+                if (lane == 0) sFlag[s] = need_mask ? 1 : 0;
+                mbar_arrive(bar_evfull(s));
+            }
+        } else if (warp == 9 && lane == 0) {
+            // ================= MMA issuer =================
+            const uint64_t dQ0 = smem_desc(sQ, 16, 1024);
+            const uint64_t dK0 = smem_desc(sKV, 16, 1024);
+            const uint64_t dV0 = smem_desc(sKV + L::TB, BOX_BYTES, 1024);
+            constexpr uint64_t TBU = (uint64_t)(L::TB >> 4);
+            auto issue_s = [&](int t, int s) {
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
+                    mma_ss(tmem + t * 128, dQ0 + t * TBU + off, dK0 + s * 2 * TBU + off, IDESC_S, kk > 0);
+                }
+                mma_commit(bar_s(t));
+            };
+            if (nlist > 0) {
+                mbar_wait(bar_q, 0, abort_flag, status);
+                mbar_wait(bar_kvfull(0), 0, abort_flag, status);
+                tc_fence_after();
+                for (int t = 0; t < ntile; ++t) issue_s(t, 0);
+            }
+            for (int i = 0; i < nlist; ++i) {
+                const int s = i & 1;
+                for (int t = 0; t < ntile; ++t) {
+                    // O_t += P_t V(i):  A = P rows from tensor memory (16 keys = 8 packed columns per step),
+                    //                   B = V, MN-major, 16 key rows per step
+                    mbar_wait(bar_p(t), i & 1, abort_flag, status);
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < TILE / 16; ++kk)
+                        mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, dV0 + s * 2 * TBU + (uint64_t)(kk * 128), IDESC_O,
+                               (i > 0) || (kk > 0));
+                    if (t == ntile - 1) mma_commit(bar_kvfree(s));      // K(i), V(i) no longer read by anything issued later
+                    if (i + 1 < nlist) {
+                        if (t == 0) {
+                            mbar_wait(bar_kvfull(s ^ 1), ((i + 1) >> 1) & 1, abort_flag, status);
+                            tc_fence_after();
+                        }
+                        issue_s(t, s ^ 1);
+                    }
+                }
+            }
+            mma_commit(bar_done);
         }
-        if (need_mask) {
-            const int j = n * TILE + tid;
-            sEv[tid] = (j < T) ? mv.evict[tok0 + j] : 0;   // 0: visible to nobody
-        }
-        if (tid == 0) {
-            if (t == 0) mbar_wait(bar_q, 0, abort_flag, status);
-            mbar_wait(bar_kv, ph, abort_flag, status);
+    } else {
+        // ================= softmax groups =================
+        reg_inc<208>();
+        const int t = warp >> 2;                                  // which query tile / head
+        if (t < ntile) {
+            const int quad = warp & 3;
+            const int row = quad * 32 + lane;                     // query row of the tile == TMEM lane
+            const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
+            const uint32_t tmem_S = tmem + t * 128 + lane_sel;
+            const uint32_t tmem_O = tmem + 256 + t * 128 + lane_sel;
+            const int h = h0 + t;
+            const int qi = m * TILE + row;                        // trace-local query index
+            float ref_max = -INFINITY;                            // base-2 domain; the exponent's reference
+            float run_sum = 0.f;
+
+            for (int i = 0; i < nlist; ++i) {
+                const int s = i & 1;
+                const int n = list[i];
+                mbar_wait(bar_evfull(s), (i >> 1) & 1, abort_flag, status);
+                const bool need_mask = sFlag[s] != 0;
+                mbar_wait(bar_s(t), i & 1, abort_flag, status);
+                tc_fence_after();
+                float sv[TILE];
+#pragma unroll
+                for (int c = 0; c < TILE / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_S + c * 32, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) sv[c * 32 + e] = __uint_as_float(r[e]) * p.scale_log2;
+                }
+                if (need_mask) {
+                    const int4* ev4 = reinterpret_cast<const int4*>(sEv + s * TILE);
+#pragma unroll
+                    for (int e4 = 0; e4 < TILE / 4; ++e4) {
+                        const int4 ev = ev4[e4];
+                        const int j = n * TILE + e4 * 4;
+                        sv[e4 * 4 + 0] = ((j + 0 <= qi) && (qi < ev.x)) ? sv[e4 * 4 + 0] : -INFINITY;
+                        sv[e4 * 4 + 1] = ((j + 1 <= qi) && (qi < ev.y)) ? sv[e4 * 4 + 1] : -INFINITY;
+                        sv[e4 * 4 + 2] = ((j + 2 <= qi) && (qi < ev.z)) ? sv[e4 * 4 + 2] : -INFINITY;
+                        sv[e4 * 4 + 3] = ((j + 3 <= qi) && (qi < ev.w)) ? sv[e4 * 4 + 3] : -INFINITY;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_evfree(s));
+                float tile_max = sv[0];
+#pragma unroll
+                for (int e = 1; e < TILE; ++e) tile_max = fmaxf(tile_max, sv[e]);
+                // lazy rescale: move the reference only when the maximum ran away from it
+                const bool grow = (tile_max > ref_max + RESCALE_THRESHOLD) || (ref_max == -INFINITY && tile_max > -INFINITY);
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float new_ref = grow ? tile_max : ref_max;
+                    const float alpha = (new_ref == -INFINITY) ? 1.f : fast_exp2(ref_max - new_ref);   // ref_max = -inf -> 0
+                    run_sum *= alpha;
+                    ref_max = new_ref;
+                    if (i > 0) {
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t r[32];
+                            tmem_ld32(tmem_O + c * 32, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+                            tmem_st32(tmem_O + c * 32, r);
+                        }
+                    }
+                }
+                const float use_ref = (ref_max == -INFINITY) ? 0.f : ref_max;
+                float tile_sum = 0.f;
+                uint32_t pk[TILE / 2];
+#pragma unroll
+                for (int e = 0; e < TILE; e += 2) {
+                    const float p0 = fast_exp2(sv[e] - use_ref);
+                    const float p1 = fast_exp2(sv[e + 1] - use_ref);
+                    tile_sum += p0 + p1;
+                    pk[e >> 1] = pack_bf16(p0, p1);
+                }
+                run_sum += tile_sum;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t r[32];
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) r[e] = pk[c * 32 + e];
+                    tmem_st32(tmem_S + c * 32, r);         // P (bf16, 64 columns) over the S columns already read
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p(t));
+            }
+
+            // ---- epilogue: O / l -> bf16, LSE -> fp32 ----
+            mbar_wait(bar_done, 0, abort_flag, status);
             tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
-                mma_ss(tmem_S, smem_desc(sQ + off, 16, 1024), smem_desc(sK + off, 16, 1024), IDESC_S, kk > 0);
-            }
-            mma_commit(bar_s);
-        }
-        __syncthreads();                       // sEv visible; also keeps the warps together
-        mbar_wait(bar_s, ph, abort_flag, status);
-        tc_fence_after();
-
-        // ---- softmax on this thread's row --------------------------------------------------
-        float sv[TILE];
-#pragma unroll
-        for (int c = 0; c < TILE / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld32(tmem_S + lane_sel + c * 32, r);
-            tmem_wait_ld();
-#pragma unroll
-            for (int e = 0; e < 32; ++e) sv[c * 32 + e] = __uint_as_float(r[e]) * p.scale_log2;
-        }
-        if (need_mask) {
-#pragma unroll
-            for (int e = 0; e < TILE; ++e) {
-                const int j = n * TILE + e;
-                const bool ok = (j <= qi) && (qi < sEv[e]);
-                sv[e] = ok ? sv[e] : -INFINITY;
-            }
-        }
-        float tile_max = sv[0];
-#pragma unroll
-        for (int e = 1; e < TILE; ++e) tile_max = fmaxf(tile_max, sv[e]);
-        const float new_max = fmaxf(run_max, tile_max);
-        const float use_max = (new_max == -INFINITY) ? 0.f : new_max;
-        const float alpha = fast_exp2(run_max - use_max);      // run_max = -inf -> 0
-        float tile_sum = 0.f;
-        uint32_t pk[TILE / 2];
-#pragma unroll
-        for (int e = 0; e < TILE; e += 2) {
-            const float p0 = fast_exp2(sv[e] - use_max);
-            const float p1 = fast_exp2(sv[e + 1] - use_max);
-            tile_sum += p0 + p1;
-            pk[e >> 1] = pack_bf16(p0, p1);
-        }
-        run_sum = run_sum * alpha + tile_sum;
-        run_max = new_max;
-        // P (bf16, 64 columns) over the S columns this thread has already read
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-            uint32_t r[32];
-#pragma unroll
-            for (int e = 0; e < 32; ++e) r[e] = pk[c * 32 + e];
-            tmem_st32(tmem_S + lane_sel + c * 32, r);
-        }
-        // rescale O when some row of the warp moved its maximum
-        if (t > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+            const bool valid = qi < T;
+            const float inv = (run_sum > 0.f && nlist > 0) ? 1.f / run_sum : 0.f;
+            __nv_bfloat16* orow = p.out + ((size_t)(tok0 + qi) * p.Hq + h) * D;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t r[32];
-                tmem_ld32(tmem_O + lane_sel + c * 32, r);
+                tmem_ld32(tmem_O + c * 32, r);
                 tmem_wait_ld();
+                if (nlist == 0) {      // only a bad evict_at (already reported by the metadata pass) gets here
 #pragma unroll
-                for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-                tmem_st32(tmem_O + lane_sel + c * 32, r);
-            }
-        }
-        tmem_wait_st();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after();
+                    for (int e = 0; e < 32; ++e) r[e] = 0u;
+                }
+                if (valid) {
+                    uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
 #pragma unroll
-            for (int kk = 0; kk < TILE / 16; ++kk) {
-                // A: P rows, 16 keys = 8 packed columns per step.  B: V, MN-major, 16 key rows per step.
-                mma_ts(tmem_O, tmem_S + kk * 8, smem_desc(sV + kk * 2048, BOX_BYTES, 1024), IDESC_O, (t > 0) || (kk > 0));
+                    for (int e = 0; e < 4; ++e) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(r[e * 8 + 0]) * inv, __uint_as_float(r[e * 8 + 1]) * inv);
+                        w.y = pack_bf16(__uint_as_float(r[e * 8 + 2]) * inv, __uint_as_float(r[e * 8 + 3]) * inv);
+                        w.z = pack_bf16(__uint_as_float(r[e * 8 + 4]) * inv, __uint_as_float(r[e * 8 + 5]) * inv);
+                        w.w = pack_bf16(__uint_as_float(r[e * 8 + 6]) * inv, __uint_as_float(r[e * 8 + 7]) * inv);
+                        dst[e] = w;
+                    }
+                }
             }
-            mma_commit(bar_o);
+            if (valid) p.lse[(size_t)h * p.total_tokens + tok0 + qi] = ref_max * 0.6931471805599453f + logf(run_sum);
         }
-        mbar_wait(bar_o, ph, abort_flag, status);   // K, V, P free again; O complete
-        tc_fence_after();
     }
-
-    // A row of blocks with no visible key block can only come from a bad evict_at (already
-    // reported by the metadata pass): drain the Q load and write zeros.
+    // a Q load whose CTA had no key block to walk is drained before the CTA leaves
     if (nlist == 0 && tid == 0) mbar_wait(bar_q, 0, abort_flag, status);
-
-    // ---- epilogue ------------------------------------------------------------------------------
-    const bool valid = qi < T;
-    const float inv = (run_sum > 0.f && nlist > 0) ? 1.f / run_sum : 0.f;
-    __nv_bfloat16* orow = p.out + ((size_t)(tok0 + qi) * p.Hq + h) * D;
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tmem_O + lane_sel + c * 32, r);
-        tmem_wait_ld();
-        if (nlist == 0) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) r[e] = 0u;
-        }
-        if (valid) {
-            uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                uint4 w;
-                w.x = pack_bf16(__uint_as_float(r[e * 8 + 0]) * inv, __uint_as_float(r[e * 8 + 1]) * inv);
-                w.y = pack_bf16(__uint_as_float(r[e * 8 + 2]) * inv, __uint_as_float(r[e * 8 + 3]) * inv);
-                w.z = pack_bf16(__uint_as_float(r[e * 8 + 4]) * inv, __uint_as_float(r[e * 8 + 5]) * inv);
-                w.w = pack_bf16(__uint_as_float(r[e * 8 + 6]) * inv, __uint_as_float(r[e * 8 + 7]) * inv);
-                dst[e] = w;
-            }
-        }
-    }
-    if (valid) p.lse[(size_t)h * p.total_tokens + tok0 + qi] = run_max * 0.6931471805599453f + logf(run_sum);
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
+    if (warp == 9) {
+        __syncwarp();
+        tmem_dealloc(tmem, TMEM_COLS);
+    }
 }
 
 template <int D>
@@ -244,8 +328,9 @@ static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
                       int nb_cap, cudaStream_t st) {
     auto kern = fwd_kernel<D>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::DYN_BYTES) != cudaSuccess) return KVS_ERR_CUDA;
-    dim3 grid(nb_cap, p.Hq, 1);
-    kern<<<grid, 128, FwdSmem<D>::DYN_BYTES, st>>>(tq, tk, tv, mv, p);
+    const int G = p.Hq / p.Hkv;
+    dim3 grid(nb_cap, p.Hkv * ((G + 1) / 2), 1);
+    kern<<<grid, FWD_THREADS, FwdSmem<D>::DYN_BYTES, st>>>(tq, tk, tv, mv, p);
     return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
 }
 

@@ -94,8 +94,8 @@ struct BwdSmem {
     static constexpr int OFF_DO = 4 * TB;            // 1 stage
     static constexpr int OFF_DS = 5 * TB;            // 128 keys x 128 queries bf16
     static constexpr int OFF_STG = OFF_DS + TILE * TILE * 2;   // 2 staging buffers for dQ chunks
-    static constexpr int OFF_LSE = OFF_STG + 2 * STG_BYTES;    // 2 stages x 128 fp32 (already * log2 e)
-    static constexpr int OFF_DVEC = OFF_LSE + 2 * TILE * 4;    // 2 stages x 128 fp32 (already * scale)
+    static constexpr int OFF_LSE = OFF_STG + 2 * STG_BYTES;    // 2 stages x 128 fp32: -lse * log2 e
+    static constexpr int OFF_DVEC = OFF_LSE + 2 * TILE * 4;    // 2 stages x 128 fp32: -D * scale
     static constexpr int OFF_BAR = OFF_DVEC + 2 * TILE * 4;
     static constexpr int OFF_MISC = OFF_BAR + 16 * 8;          // tmem base, abort flag
     static constexpr int TOTAL = OFF_MISC + 16;
@@ -175,7 +175,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     auto bar_ldfull = [&](int s) { return bars + 8 * (3 + s); };
     auto bar_qfree = [&](int s) { return bars + 8 * (5 + s); };
     const uint32_t bar_dofull = bars + 8 * 7, bar_dofree = bars + 8 * 8, bar_s = bars + 8 * 9, bar_dp = bars + 8 * 10,
-                   bar_p = bars + 8 * 11, bar_ds = bars + 8 * 12, bar_dq = bars + 8 * 13, bar_drained = bars + 8 * 14;
+                   bar_p = bars + 8 * 11, bar_ds = bars + 8 * 12, bar_dq = bars + 8 * 13, bar_drained = bars + 8 * 14,
+                   bar_dss = bars + 8 * 15;
 
     if (tid == 0) {
         *abort_flag = 0;
@@ -191,6 +192,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         mbar_init(bar_dp, 1);
         mbar_init(bar_p, 8);
         mbar_init(bar_ds, 8);
+        mbar_init(bar_dss, 8);
         mbar_init(bar_dq, 1);
         mbar_init(bar_drained, 4);
         fence_mbar_init();
@@ -235,9 +237,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 for (int u = 0; u < 4; ++u) {
                     const int i = lane * 4 + u;
                     const bool qv = (m * TILE + i) < T;
-                    // +inf makes P vanish for the rows past the end of the trace
-                    sLse[s * TILE + i] = qv ? p.lse[rowbase + i] * 1.4426950408889634f : INFINITY;
-                    sDv[s * TILE + i] = qv ? p.dvec[rowbase + i] * p.scale : 0.f;
+                    // stored negated (they are subtracted with one fused multiply-add); -inf makes P vanish
+                    // for the rows past the end of the trace
+                    sLse[s * TILE + i] = qv ? p.lse[rowbase + i] * -1.4426950408889634f : -INFINITY;
+                    sDv[s * TILE + i] = qv ? p.dvec[rowbase + i] * -p.scale : 0.f;
                 }
                 mbar_arrive(bar_ldfull(s));
                 // dO(j): single buffer, free once dP(j-1) and dV(j-1) have completed
@@ -312,6 +315,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 for (int kk = 0; kk < TILE / 16; ++kk)
                     mma_ts(tmem_dK, tmem_P + (kk >> 2) * 64 + (kk & 3) * 8, dQ_mn + so + (uint64_t)(kk * 128), IDESC_KV,
                            (j > 0) || (kk > 0));
+                mbar_wait(bar_dss, ph, abort_flag, status);
 #pragma unroll
                 for (int kk = 0; kk < TILE / 16; ++kk)
                     mma_ss(tmem_P, dDS_mn + (uint64_t)(kk * 128), dK_mn + (uint64_t)(kk * 128), IDESC_DQ, kk > 0);
@@ -386,7 +390,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         auto phase_p = [&](int j) {        // P^T(j) = exp2(S^T * c - lse), masked
             const int s = j & 1;
             const int m = n + j % nm;
-            const bool need_mask = (cls_next != KVS_CLASS_FULL) || key_tail;
+            const bool need_mask = (cls_next != KVS_CLASS_FULL) || key_tail || (m * TILE + TILE > T);
             if (j + 1 < n_iter) cls_next = cls_col[(size_t)(n + (j + 1) % nm) * nb];
             mbar_wait(bar_ldfull(s), (j >> 1) & 1, abort_flag, status);
             mbar_wait(bar_s, j & 1, abort_flag, status);
@@ -397,27 +401,23 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             tmem_ld32(tmem_S + lane_sel + col0, r0);
             tmem_ld32(tmem_S + lane_sel + col0 + 32, r1);
             tmem_wait_ld();
+            const float2 c2 = make_float2(p.scale_log2, p.scale_log2);
 #pragma unroll
-            for (int e4 = 0; e4 < 8; ++e4) {
+            for (int e4 = 0; e4 < 16; ++e4) {          // packed fp32x2 multiply-adds, then one ex2 per element
                 const float4 l = l4[e4];
-                pv[e4 * 4 + 0] = fast_exp2(fmaf(__uint_as_float(r0[e4 * 4 + 0]), p.scale_log2, -l.x));
-                pv[e4 * 4 + 1] = fast_exp2(fmaf(__uint_as_float(r0[e4 * 4 + 1]), p.scale_log2, -l.y));
-                pv[e4 * 4 + 2] = fast_exp2(fmaf(__uint_as_float(r0[e4 * 4 + 2]), p.scale_log2, -l.z));
-                pv[e4 * 4 + 3] = fast_exp2(fmaf(__uint_as_float(r0[e4 * 4 + 3]), p.scale_log2, -l.w));
-            }
-#pragma unroll
-            for (int e4 = 0; e4 < 8; ++e4) {
-                const float4 l = l4[8 + e4];
-                pv[32 + e4 * 4 + 0] = fast_exp2(fmaf(__uint_as_float(r1[e4 * 4 + 0]), p.scale_log2, -l.x));
-                pv[32 + e4 * 4 + 1] = fast_exp2(fmaf(__uint_as_float(r1[e4 * 4 + 1]), p.scale_log2, -l.y));
-                pv[32 + e4 * 4 + 2] = fast_exp2(fmaf(__uint_as_float(r1[e4 * 4 + 2]), p.scale_log2, -l.z));
-                pv[32 + e4 * 4 + 3] = fast_exp2(fmaf(__uint_as_float(r1[e4 * 4 + 3]), p.scale_log2, -l.w));
+                const uint32_t* r = (e4 < 8) ? &r0[e4 * 4] : &r1[(e4 - 8) * 4];
+                const float2 x01 = __ffma2_rn(make_float2(__uint_as_float(r[0]), __uint_as_float(r[1])), c2, make_float2(l.x, l.y));
+                const float2 x23 = __ffma2_rn(make_float2(__uint_as_float(r[2]), __uint_as_float(r[3])), c2, make_float2(l.z, l.w));
+                pv[e4 * 4 + 0] = fast_exp2(x01.x);
+                pv[e4 * 4 + 1] = fast_exp2(x01.y);
+                pv[e4 * 4 + 2] = fast_exp2(x23.x);
+                pv[e4 * 4 + 3] = fast_exp2(x23.y);
             }
             if (need_mask) {
 #pragma unroll
                 for (int e = 0; e < 64; ++e) {
                     const int qi = m * TILE + col0 + e;
-                    pv[e] = ((kj <= qi) && (qi < my_ev)) ? pv[e] : 0.f;
+                    pv[e] = ((kj <= qi) && (qi < my_ev) && (qi < T)) ? pv[e] : 0.f;
                 }
             }
             uint32_t pk[32];
@@ -441,22 +441,19 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             tmem_ld32(tmem_P + lane_sel + col0, r0);
             tmem_ld32(tmem_P + lane_sel + col0 + 32, r1);
             tmem_wait_ld();
+            if (tid == 0) KVS_TR(2, j, 14);
             uint32_t dk_[32];
+            const float2 sc2 = make_float2(p.scale, p.scale);
 #pragma unroll
-            for (int e4 = 0; e4 < 8; ++e4) {
+            for (int e4 = 0; e4 < 16; ++e4) {          // dS = P * (scale dP - scale D), two elements per instruction
                 const float4 dd = d4[e4];
-                dk_[e4 * 2 + 0] = pack_bf16(pv[e4 * 4 + 0] * fmaf(__uint_as_float(r0[e4 * 4 + 0]), p.scale, -dd.x),
-                                           pv[e4 * 4 + 1] * fmaf(__uint_as_float(r0[e4 * 4 + 1]), p.scale, -dd.y));
-                dk_[e4 * 2 + 1] = pack_bf16(pv[e4 * 4 + 2] * fmaf(__uint_as_float(r0[e4 * 4 + 2]), p.scale, -dd.z),
-                                           pv[e4 * 4 + 3] * fmaf(__uint_as_float(r0[e4 * 4 + 3]), p.scale, -dd.w));
-            }
-#pragma unroll
-            for (int e4 = 0; e4 < 8; ++e4) {
-                const float4 dd = d4[8 + e4];
-                dk_[16 + e4 * 2 + 0] = pack_bf16(pv[32 + e4 * 4 + 0] * fmaf(__uint_as_float(r1[e4 * 4 + 0]), p.scale, -dd.x),
-                                                pv[32 + e4 * 4 + 1] * fmaf(__uint_as_float(r1[e4 * 4 + 1]), p.scale, -dd.y));
-                dk_[16 + e4 * 2 + 1] = pack_bf16(pv[32 + e4 * 4 + 2] * fmaf(__uint_as_float(r1[e4 * 4 + 2]), p.scale, -dd.z),
-                                                pv[32 + e4 * 4 + 3] * fmaf(__uint_as_float(r1[e4 * 4 + 3]), p.scale, -dd.w));
+                const uint32_t* r = (e4 < 8) ? &r0[e4 * 4] : &r1[(e4 - 8) * 4];
+                const float2 t01 = __ffma2_rn(make_float2(__uint_as_float(r[0]), __uint_as_float(r[1])), sc2, make_float2(dd.x, dd.y));
+                const float2 t23 = __ffma2_rn(make_float2(__uint_as_float(r[2]), __uint_as_float(r[3])), sc2, make_float2(dd.z, dd.w));
+                const float2 d01 = __fmul2_rn(make_float2(pv[e4 * 4 + 0], pv[e4 * 4 + 1]), t01);
+                const float2 d23 = __fmul2_rn(make_float2(pv[e4 * 4 + 2], pv[e4 * 4 + 3]), t23);
+                dk_[e4 * 2 + 0] = pack_bf16(d01.x, d01.y);
+                dk_[e4 * 2 + 1] = pack_bf16(d23.x, d23.y);
             }
             tmem_st32(tmem_P + lane_sel + col0, dk_);
             // dS^T row -> shared memory, MN-major (queries contiguous), 128-byte swizzle: the 64 queries of
@@ -465,11 +462,14 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             for (int c = 0; c < 8; ++c)
                 *reinterpret_cast<uint4*>(sDS_row + ((c ^ (row & 7)) << 4)) =
                     make_uint4(dk_[c * 4], dk_[c * 4 + 1], dk_[c * 4 + 2], dk_[c * 4 + 3]);
-            tmem_wait_st();
-            fence_proxy_async();
+            if (tid == 0) KVS_TR(2, j, 15);
+            tmem_wait_st();                          // dS^T in tensor memory: dK can start
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_ds);
+            fence_proxy_async();                     // dS in shared memory: dQ can start
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_dss);
             if (tid == 0) KVS_TR(2, j, 13);
         };
 

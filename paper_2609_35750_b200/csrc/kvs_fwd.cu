@@ -213,14 +213,22 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 const bool need_mask = sFlag[s] != 0;
                 mbar_wait(bar_s(t), i & 1, abort_flag, status);
                 tc_fence_after();
+                // raw logits of this row (the softmax scale is positive, so the maximum can be taken before it)
                 float sv[TILE];
-#pragma unroll
-                for (int c = 0; c < TILE / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem_S + c * 32, r);
+                {
+                    uint32_t r0[32], r1[32], r2[32], r3[32];
+                    tmem_ld32(tmem_S, r0);
+                    tmem_ld32(tmem_S + 32, r1);
+                    tmem_ld32(tmem_S + 64, r2);
+                    tmem_ld32(tmem_S + 96, r3);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) sv[c * 32 + e] = __uint_as_float(r[e]) * p.scale_log2;
+                    for (int e = 0; e < 32; ++e) {
+                        sv[e] = __uint_as_float(r0[e]);
+                        sv[32 + e] = __uint_as_float(r1[e]);
+                        sv[64 + e] = __uint_as_float(r2[e]);
+                        sv[96 + e] = __uint_as_float(r3[e]);
+                    }
                 }
                 if (need_mask) {
                     const int4* ev4 = reinterpret_cast<const int4*>(sEv + s * TILE);
@@ -236,9 +244,17 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_evfree(s));
-                float tile_max = sv[0];
+                // eight independent partial maxima, then a short tree (no 127-deep dependency chain)
+                float mx[8];
 #pragma unroll
-                for (int e = 1; e < TILE; ++e) tile_max = fmaxf(tile_max, sv[e]);
+                for (int u = 0; u < 8; ++u) mx[u] = sv[u];
+#pragma unroll
+                for (int e = 8; e < TILE; e += 8) {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) mx[u] = fmaxf(mx[u], sv[e + u]);
+                }
+                const float tile_max =
+                    fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
                 // lazy rescale: move the reference only when the maximum ran away from it
                 const bool grow = (tile_max > ref_max + RESCALE_THRESHOLD) || (ref_max == -INFINITY && tile_max > -INFINITY);
                 if (__any_sync(0xffffffffu, grow)) {
@@ -258,16 +274,24 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         }
                     }
                 }
-                const float use_ref = (ref_max == -INFINITY) ? 0.f : ref_max;
-                float tile_sum = 0.f;
+                const float neg_ref = (ref_max == -INFINITY) ? 0.f : -ref_max;
+                // packed fp32x2: one multiply-add forms two exponents, one add accumulates two terms
+                const float2 c2 = make_float2(p.scale_log2, p.scale_log2);
+                const float2 nr2 = make_float2(neg_ref, neg_ref);
+                float2 ts[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 uint32_t pk[TILE / 2];
 #pragma unroll
-                for (int e = 0; e < TILE; e += 2) {
-                    const float p0 = fast_exp2(sv[e] - use_ref);
-                    const float p1 = fast_exp2(sv[e + 1] - use_ref);
-                    tile_sum += p0 + p1;
-                    pk[e >> 1] = pack_bf16(p0, p1);
+                for (int e = 0; e < TILE; e += 8) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float2 x = __ffma2_rn(make_float2(sv[e + 2 * u], sv[e + 2 * u + 1]), c2, nr2);
+                        const float2 pp = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                        ts[u] = __fadd2_rn(ts[u], pp);
+                        pk[(e >> 1) + u] = pack_bf16(pp.x, pp.y);
+                    }
                 }
+                const float2 t01 = __fadd2_rn(ts[0], ts[1]), t23 = __fadd2_rn(ts[2], ts[3]);
+                const float tile_sum = (t01.x + t01.y) + (t23.x + t23.y);
                 run_sum += tile_sum;
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {

@@ -74,10 +74,10 @@ __global__ void bwd_cast_kernel(const float* __restrict__ acc, __nv_bfloat16* __
 // Registers are re-balanced per warp group with setmaxnreg (compute 144, drain 136, the rest 88).
 //
 // Tensor memory (512 columns):  [0,128) S^T fp32, then P^T bf16 in [0,32) and [64,96)
-//                               [128,256) dP^T fp32, then dS^T bf16 in +[0,32), +[64,96); then dQ fp32
+//                               [128,256) dP^T fp32, then dQ fp32
 //                               [256,256+D) dV     [384,384+D) dK
 // Per iteration j (one (head, query block) tile) the tensor pipe runs, in this order,
-//     dP^T(j) = V dO^T,  dV(j) += P^T dO,  S^T(j+1) = K Q^T,  dK(j) += dS^T Q,  dQ(j) = dS K
+//     dP^T(j) = V dO^T,  dV(j) += P^T dO,  S^T(j+1) = K Q^T,  dQ(j) = dS K,  dK(j) += dS^T Q
 // while the compute warps run  dS(j), P(j+1)  and the drain warps empty dQ(j).  The softmax scale
 // is folded into dS (dS = P (scale dP - scale D)), so dK and dQ leave the tensor core scaled.
 // Rows of a dQ tile past the end of a trace are exactly zero (their P is zero), so the reduce-add
@@ -175,7 +175,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     auto bar_ldfull = [&](int s) { return bars + 8 * (3 + s); };
     auto bar_qfree = [&](int s) { return bars + 8 * (5 + s); };
     const uint32_t bar_dofull = bars + 8 * 7, bar_dofree = bars + 8 * 8, bar_s = bars + 8 * 9, bar_dp = bars + 8 * 10,
-                   bar_p = bars + 8 * 11, bar_ds = bars + 8 * 12, bar_dq = bars + 8 * 13, bar_drained = bars + 8 * 14,
+                   bar_p = bars + 8 * 11, bar_dq = bars + 8 * 13, bar_drained = bars + 8 * 14,
                    bar_dss = bars + 8 * 15;
 
     if (tid == 0) {
@@ -191,7 +191,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         mbar_init(bar_s, 1);
         mbar_init(bar_dp, 1);
         mbar_init(bar_p, 8);
-        mbar_init(bar_ds, 8);
         mbar_init(bar_dss, 8);
         mbar_init(bar_dq, 1);
         mbar_init(bar_drained, 4);
@@ -257,6 +256,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const uint64_t dK_k = smem_desc(sK, 16, 1024), dV_k = smem_desc(sV, 16, 1024);
             const uint64_t dQ_k = smem_desc(sQ, 16, 1024), dDO_k = smem_desc(sDO, 16, 1024);
             const uint64_t dK_mn = smem_desc(sK, BOX_BYTES, 1024), dDS_mn = smem_desc(sDS, BOX_BYTES, 1024);
+            const uint64_t dDS_k = smem_desc(sDS, 16, 1024);
             const uint64_t dQ_mn = smem_desc(sQ, BOX_BYTES, 1024), dDO_mn = smem_desc(sDO, BOX_BYTES, 1024);
             constexpr uint64_t STAGE = (uint64_t)(L::TB >> 4);
             mbar_wait(bar_kv, 0, abort_flag, status);
@@ -307,19 +307,21 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     }
                     mma_commit(bar_s);
                 }
-                // dK(j) += dS^T Q, then dQ(j) = dS K (dQ overwrites the columns that hold dS^T, so it goes last)
-                mbar_wait(bar_ds, ph, abort_flag, status);
+                // dQ(j) = dS K, then dK(j) += dS^T Q.  Both read dS from shared memory: the same swizzled buffer
+                // is the MN-major A operand of dQ (queries contiguous) and, read as [keys x queries] rows, the
+                // K-major A operand of dK; dQ goes first so that the drain can start while dK still runs.
+                mbar_wait(bar_dss, ph, abort_flag, status);
                 tc_fence_after();
                 KVS_TR(0, j, 6);
 #pragma unroll
                 for (int kk = 0; kk < TILE / 16; ++kk)
-                    mma_ts(tmem_dK, tmem_P + (kk >> 2) * 64 + (kk & 3) * 8, dQ_mn + so + (uint64_t)(kk * 128), IDESC_KV,
-                           (j > 0) || (kk > 0));
-                mbar_wait(bar_dss, ph, abort_flag, status);
-#pragma unroll
-                for (int kk = 0; kk < TILE / 16; ++kk)
                     mma_ss(tmem_P, dDS_mn + (uint64_t)(kk * 128), dK_mn + (uint64_t)(kk * 128), IDESC_DQ, kk > 0);
                 mma_commit(bar_dq);
+#pragma unroll
+                for (int kk = 0; kk < TILE / 16; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
+                    mma_ss(tmem_dK, dDS_k + off, dQ_mn + so + (uint64_t)(kk * 128), IDESC_KV, (j > 0) || (kk > 0));
+                }
                 mma_commit(bar_qfree(s));
                 KVS_TR(0, j, 7);
             }
@@ -455,7 +457,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 dk_[e4 * 2 + 0] = pack_bf16(d01.x, d01.y);
                 dk_[e4 * 2 + 1] = pack_bf16(d23.x, d23.y);
             }
-            tmem_st32(tmem_P + lane_sel + col0, dk_);
             // dS^T row -> shared memory, MN-major (queries contiguous), 128-byte swizzle: the 64 queries of
             // this half are the 128-byte row `row` of block `half`; 16-byte chunk c sits at (c ^ (row % 8))
 #pragma unroll
@@ -463,11 +464,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 *reinterpret_cast<uint4*>(sDS_row + ((c ^ (row & 7)) << 4)) =
                     make_uint4(dk_[c * 4], dk_[c * 4 + 1], dk_[c * 4 + 2], dk_[c * 4 + 3]);
             if (tid == 0) KVS_TR(2, j, 15);
-            tmem_wait_st();                          // dS^T in tensor memory: dK can start
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_ds);
-            fence_proxy_async();                     // dS in shared memory: dQ can start
+            fence_proxy_async();                     // dS visible to the tensor core's reads of shared memory
+            tc_fence_before();                       // orders this thread's reads of dP^T before the dQ MMA that overwrites it
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_dss);
             if (tid == 0) KVS_TR(2, j, 13);

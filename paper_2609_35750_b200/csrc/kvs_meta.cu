@@ -128,7 +128,7 @@ __global__ void meta_classify_kernel(MetaHeader* hdr, const int32_t* __restrict_
 // ---- kernel 3: work orders, heaviest first (bucket sort, one CTA per order) -------------------
 // blockIdx.x = 0: query blocks by their number of non-empty key blocks (forward);
 // blockIdx.x = 1: key blocks by the length of their query-block range (backward).
-// Only the launch order of work depends on it; ties may land in any order.
+// Only the launch order of work depends on it; ties keep their order in the batch.
 constexpr int ORDER_BINS = 4096;
 __global__ void __launch_bounds__(1024)
 meta_order_kernel(MetaHeader* hdr, const int32_t* __restrict__ blk_off, const int32_t* __restrict__ blk_trace,
@@ -140,8 +140,10 @@ meta_order_kernel(MetaHeader* hdr, const int32_t* __restrict__ blk_off, const in
     const bool bwd = blockIdx.x == 1;
     int32_t* order = bwd ? bwd_order : fwd_order;
     auto key = [&](int i) {
+        // coarse buckets (16 tiles): exact lengths would interleave blocks from all over the batch,
+        // coarse ones keep runs of neighbouring blocks together while still starting the long ones first
         const int k = bwd ? (col_last[i] - (i - blk_off[blk_trace[i]]) + 1) : row_cnt[i];
-        return min(max(k, 0), ORDER_BINS - 1);
+        return min(max(k >> 4, 0), ORDER_BINS - 1);
     };
     for (int i = threadIdx.x; i < ORDER_BINS; i += blockDim.x) bins[i] = 0;
     __syncthreads();
@@ -180,7 +182,19 @@ meta_order_kernel(MetaHeader* hdr, const int32_t* __restrict__ blk_off, const in
         run += c[u];
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < n; i += blockDim.x) order[atomicAdd(&bins[key(i)], 1)] = i;
+    // Stable scatter by one warp, 32 blocks at a time in index order: blocks with equal keys keep their
+    // order in the trace, so CTAs launched together work on neighbouring blocks and share tiles in L2.
+    if (warp == 0) {
+        for (int i0 = 0; i0 < n; i0 += 32) {
+            const int i = i0 + lane;
+            const int k = (i < n) ? key(i) : -1;
+            const unsigned same = __match_any_sync(0xffffffffu, k);
+            if (i < n) order[bins[k] + __popc(same & ((1u << lane) - 1u))] = i;
+            __syncwarp();
+            if (i < n && lane == (__ffs(same) - 1)) bins[k] += __popc(same);
+            __syncwarp();
+        }
+    }
 }
 
 }  // namespace kvs

@@ -172,11 +172,14 @@ __device__ __forceinline__ uint32_t mbar_try_wait_hint(uint32_t bar, uint32_t pa
         : "memory");
     return ok;
 }
+#ifndef KVS_WAIT_HINT_NS
+#define KVS_WAIT_HINT_NS 20000u
+#endif
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
     if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
     while (true) {
-        if (mbar_try_wait_hint(bar, parity, 20000u)) return;
+        if (mbar_try_wait_hint(bar, parity, KVS_WAIT_HINT_NS)) return;
         if (*abort_flag) return;
         if (clock64() - t0 > WAIT_LIMIT_CLOCKS) {
             *abort_flag = 1;

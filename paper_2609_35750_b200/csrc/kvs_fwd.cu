@@ -31,7 +31,7 @@ struct FwdSmem {
     static constexpr int OFF_BAR = OFF_FLAG + 16;
     static constexpr int OFF_MISC = OFF_BAR + 16 * 8;
     static constexpr int TOTAL = OFF_MISC + 16;
-    static constexpr int DYN_BYTES = TOTAL + 1024;       // slack for the 1024-byte alignment
+    static constexpr int DYN_BYTES = TOTAL + 1024 + 1024;   // slack for the 1024-byte alignment (+ room for a debug trace)
 };
 
 struct FwdParams {
@@ -40,6 +40,14 @@ struct FwdParams {
     __nv_bfloat16* out;
     float* lse;
 };
+
+#ifdef KVS_TRACE
+// Debug build only: clock64 timestamps of one CTA's pipeline events.
+__device__ long long g_trace_fwd[1024];
+#define KVS_TRF(i, ev) do { if ((i) >= 8 && (i) < 20) s_tr[((i) - 8) * 16 + (ev)] = (uint32_t)clock64(); } while (0)
+#else
+#define KVS_TRF(i, ev) do { } while (0)
+#endif
 
 template <int D>
 __global__ void __launch_bounds__(FWD_THREADS, 1)
@@ -82,6 +90,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     volatile int32_t* sFlag = reinterpret_cast<volatile int32_t*>(sgen + L::OFF_FLAG);
     uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(sgen + L::OFF_MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + L::OFF_MISC + 4);
+#ifdef KVS_TRACE
+    volatile uint32_t* s_tr = reinterpret_cast<volatile uint32_t*>(sgen + L::TOTAL);
+#endif
     const uint32_t bars = sbase + L::OFF_BAR;
     const uint32_t bar_q = bars;
     auto bar_kvfull = [&](int s) { return bars + 8 * (1 + s); };    // TMA bytes of K and V
@@ -173,8 +184,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 for (int t = 0; t < ntile; ++t) {
                     // O_t += P_t V(i):  A = P rows from tensor memory (16 keys = 8 packed columns per step),
                     //                   B = V, MN-major, 16 key rows per step
+                    KVS_TRF(i, t * 4 + 0);
                     mbar_wait(bar_p(t), i & 1, abort_flag, status);
                     tc_fence_after();
+                    KVS_TRF(i, t * 4 + 1);
 #pragma unroll
                     for (int kk = 0; kk < TILE / 16; ++kk)
                         mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, dV0 + s * 2 * TBU + (uint64_t)(kk * 128), IDESC_O,
@@ -187,6 +200,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         }
                         issue_s(t, s ^ 1);
                     }
+                    KVS_TRF(i, t * 4 + 2);
                 }
             }
             mma_commit(bar_done);
@@ -213,6 +227,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 const bool need_mask = sFlag[s] != 0;
                 mbar_wait(bar_s(t), i & 1, abort_flag, status);
                 tc_fence_after();
+                if (tid == 0) KVS_TRF(i, 8);
+                if (tid == 128) KVS_TRF(i, 13);
                 // raw logits of this row (the softmax scale is positive, so the maximum can be taken before it)
                 float sv[TILE];
                 {
@@ -230,6 +246,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         sv[96 + e] = __uint_as_float(r3[e]);
                     }
                 }
+                if (tid == 0) KVS_TRF(i, 9);
                 if (need_mask) {
                     const int4* ev4 = reinterpret_cast<const int4*>(sEv + s * TILE);
 #pragma unroll
@@ -274,6 +291,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         }
                     }
                 }
+                if (tid == 0) KVS_TRF(i, 10);
                 const float neg_ref = (ref_max == -INFINITY) ? 0.f : -ref_max;
                 // packed fp32x2: one multiply-add forms two exponents, one add accumulates two terms
                 const float2 c2 = make_float2(p.scale_log2, p.scale_log2);
@@ -292,6 +310,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 }
                 const float2 t01 = __fadd2_rn(ts[0], ts[1]), t23 = __fadd2_rn(ts[2], ts[3]);
                 const float tile_sum = (t01.x + t01.y) + (t23.x + t23.y);
+                if (tid == 0) KVS_TRF(i, 11);
                 run_sum += tile_sum;
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
@@ -304,6 +323,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p(t));
+                if (tid == 0) KVS_TRF(i, 12);
+                if (tid == 128) KVS_TRF(i, 14);
             }
 
             // ---- epilogue: O / l -> bf16, LSE -> fp32 ----
@@ -341,6 +362,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     if (nlist == 0 && tid == 0) mbar_wait(bar_q, 0, abort_flag, status);
     tc_fence_before();
     __syncthreads();
+#ifdef KVS_TRACE
+    if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 192) g_trace_fwd[tid] = s_tr[tid];
+#endif
     if (warp == 9) {
         __syncwarp();
         tmem_dealloc(tmem, TMEM_COLS);
@@ -392,3 +416,9 @@ extern "C" int kvs_attn_fwd(const void* q, const void* k, const void* v, const v
     cudaStream_t st = (cudaStream_t)stream;
     return head_dim == 64 ? launch_fwd<64>(tq, tk, tv, mv, p, L.nb_cap, st) : launch_fwd<128>(tq, tk, tv, mv, p, L.nb_cap, st);
 }
+
+#ifdef KVS_TRACE
+extern "C" int kvs_debug_read_trace_fwd(long long* host, int n) {
+    return cudaMemcpyFromSymbol(host, kvs::g_trace_fwd, sizeof(long long) * n) == cudaSuccess ? 0 : -1;
+}
+#endif

@@ -179,6 +179,9 @@ size_t kvs_host_arena_bytes(int batch, int total_tokens, int max_seqlen,
  * backward, copies out, lse, dq, dk, dv back, and SYNCHRONISES the stream.  Host buffers
  * should be page-locked for the copies to be asynchronous.  arena: device memory the caller
  * provides, >= kvs_host_arena_bytes(...), 256-byte aligned.  Returns the device status.
+ * The copy of dout overlaps the forward and the copies of out and lse overlap the backward, on an
+ * internal stream that (with four events) is created and destroyed inside the call; no device memory
+ * is allocated.
  */
 int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t* cu_seqlens_host,
                           const void* q_host, const void* k_host, const void* v_host,

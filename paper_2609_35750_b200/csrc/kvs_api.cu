@@ -148,30 +148,63 @@ extern "C" int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t
     if (arena_bytes < A.total) return KVS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     char* a = (char*)arena;
-#define KVS_CP(dst, src, bytes, kind) \
-    if (cudaMemcpyAsync(dst, src, bytes, kind, st) != cudaSuccess) return KVS_ERR_CUDA
-    KVS_CP(a + A.evict, evict_at_host, (size_t)total_tokens * 4, cudaMemcpyHostToDevice);
-    KVS_CP(a + A.cu, cu_seqlens_host, (size_t)(batch + 1) * 4, cudaMemcpyHostToDevice);
-    KVS_CP(a + A.q, q_host, A.nq_bytes, cudaMemcpyHostToDevice);
-    KVS_CP(a + A.k, k_host, A.nkv_bytes, cudaMemcpyHostToDevice);
-    KVS_CP(a + A.v, v_host, A.nkv_bytes, cudaMemcpyHostToDevice);
-    KVS_CP(a + A.dout, dout_host, A.nq_bytes, cudaMemcpyHostToDevice);
+    // A second stream carries the copies that can overlap compute (PCIe is full duplex): dout goes in
+    // while the forward runs, out and lse come back while the backward runs.  Stream and events live
+    // for this call only.
+    cudaStream_t cp = nullptr;
+    cudaEvent_t ev_in = nullptr, ev_fwd = nullptr, ev_dout = nullptr, ev_out = nullptr;
+    struct Cleanup {
+        cudaStream_t& cp;
+        cudaEvent_t &e0, &e1, &e2, &e3;
+        ~Cleanup() {
+            if (e0) cudaEventDestroy(e0);
+            if (e1) cudaEventDestroy(e1);
+            if (e2) cudaEventDestroy(e2);
+            if (e3) cudaEventDestroy(e3);
+            if (cp) cudaStreamDestroy(cp);
+        }
+    } cleanup{cp, ev_in, ev_fwd, ev_dout, ev_out};
+    if (cudaStreamCreateWithFlags(&cp, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&ev_in, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ev_fwd, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ev_dout, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ev_out, cudaEventDisableTiming) != cudaSuccess)
+        return KVS_ERR_CUDA;
+#define KVS_CP(strm, dst, src, bytes, kind) \
+    if (cudaMemcpyAsync(dst, src, bytes, kind, strm) != cudaSuccess) return KVS_ERR_CUDA
+#define KVS_CK(call) \
+    if ((call) != cudaSuccess) return KVS_ERR_CUDA
+    KVS_CP(st, a + A.evict, evict_at_host, (size_t)total_tokens * 4, cudaMemcpyHostToDevice);
+    KVS_CP(st, a + A.cu, cu_seqlens_host, (size_t)(batch + 1) * 4, cudaMemcpyHostToDevice);
+    KVS_CP(st, a + A.q, q_host, A.nq_bytes, cudaMemcpyHostToDevice);
+    KVS_CP(st, a + A.k, k_host, A.nkv_bytes, cudaMemcpyHostToDevice);
+    KVS_CP(st, a + A.v, v_host, A.nkv_bytes, cudaMemcpyHostToDevice);
+    KVS_CK(cudaEventRecord(ev_in, st));                       // dout follows q, k, v on the wire (they are needed first)
+    KVS_CK(cudaStreamWaitEvent(cp, ev_in, 0));
+    KVS_CP(cp, a + A.dout, dout_host, A.nq_bytes, cudaMemcpyHostToDevice);      // overlaps the forward
+    KVS_CK(cudaEventRecord(ev_dout, cp));
     int rc = kvs_mask_meta((const int32_t*)(a + A.evict), (const int32_t*)(a + A.cu), batch, total_tokens, max_seqlen, a + A.meta,
                            A.meta_bytes, stream);
     if (rc != KVS_OK) return rc;
     rc = kvs_attn_fwd(a + A.q, a + A.k, a + A.v, a + A.meta, batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, softmax_scale,
                       a + A.out, (float*)(a + A.lse), stream);
     if (rc != KVS_OK) return rc;
+    KVS_CK(cudaEventRecord(ev_fwd, st));
+    KVS_CK(cudaStreamWaitEvent(cp, ev_fwd, 0));
+    KVS_CP(cp, out_host, a + A.out, A.nq_bytes, cudaMemcpyDeviceToHost);         // overlaps the backward
+    KVS_CP(cp, lse_host, a + A.lse, A.lse_bytes, cudaMemcpyDeviceToHost);
+    KVS_CK(cudaEventRecord(ev_out, cp));
+    KVS_CK(cudaStreamWaitEvent(st, ev_dout, 0));
     rc = kvs_attn_bwd(a + A.dout, a + A.q, a + A.k, a + A.v, a + A.out, (const float*)(a + A.lse), a + A.meta, batch, total_tokens,
                       max_seqlen, Hq, Hkv, head_dim, softmax_scale, grad_dtype, a + A.dq, a + A.dk, a + A.dv, a + A.ws, A.ws_bytes,
                       stream);
     if (rc != KVS_OK) return rc;
-    KVS_CP(out_host, a + A.out, A.nq_bytes, cudaMemcpyDeviceToHost);
-    KVS_CP(lse_host, a + A.lse, A.lse_bytes, cudaMemcpyDeviceToHost);
-    KVS_CP(dq_host, a + A.dq, A.gq_bytes, cudaMemcpyDeviceToHost);
-    KVS_CP(dk_host, a + A.dk, A.gkv_bytes, cudaMemcpyDeviceToHost);
-    KVS_CP(dv_host, a + A.dv, A.gkv_bytes, cudaMemcpyDeviceToHost);
+    KVS_CP(st, dq_host, a + A.dq, A.gq_bytes, cudaMemcpyDeviceToHost);
+    KVS_CP(st, dk_host, a + A.dk, A.gkv_bytes, cudaMemcpyDeviceToHost);
+    KVS_CP(st, dv_host, a + A.dv, A.gkv_bytes, cudaMemcpyDeviceToHost);
+    KVS_CK(cudaStreamWaitEvent(st, ev_out, 0));               // the caller's stream ends after every copy
 #undef KVS_CP
+#undef KVS_CK
     int32_t hm[2] = {0, 0}, hw[2] = {0, 0};
     if (cudaMemcpyAsync(hm, a + A.meta, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVS_ERR_CUDA;
     if (cudaMemcpyAsync(hw, a + A.ws, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVS_ERR_CUDA;

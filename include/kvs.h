@@ -64,6 +64,17 @@ const char* kvs_strerror(int code);
 size_t kvs_mask_meta_bytes(int batch, int total_tokens, int max_seqlen);
 
 /*
+ * Compaction event log -> evict_at (Sec. 2: a compaction deletes a span of the context; the trainer
+ * masks that span from then on).  events: int32 [n_events, 4] rows (trace, when, start, end), trace-local
+ * token indices: at step `when` the keys [start, end) of that trace leave the cache.  evict_at
+ * [total_tokens] is overwritten: 2^31-1 where no event applies, else the earliest `when`.  Spans are
+ * clipped to their trace; rows naming a trace outside [0, batch) are ignored.  Whether the result
+ * satisfies evict_at[j] > j is checked by kvs_mask_meta.
+ */
+int kvs_evict_at_from_events(const int32_t* events, int n_events, const int32_t* cu_seqlens,
+                             int batch, int total_tokens, int32_t* evict_at, kvs_stream_t stream);
+
+/*
  * Mask metadata (the tile classification that lets the attention kernels skip evicted spans;
  * the paper states only that the deleted span is masked, Sec. 2 -- the tiling is this
  * library's).  For every key block n of every trace: kmin/kmax of evict_at over its valid

@@ -26,7 +26,7 @@ What it states, and where that comes from:
   force classification from the dense boolean mask.
 
 Everything is fp64 on inputs that were already rounded to bf16 by the caller.
-Pins (tests/test_oracle_pins.py): two-route agreement, no-eviction == plain
+Pins (tests/test_oracle_pins.py, tests/test_mask_families.py): two-route agreement, no-eviction == plain
 causal attention (torch's CPU scaled_dot_product_attention in fp64), softmax
 rows summing to one, central finite differences for dQ/dK/dV, zero-query
 closed forms (exp(LSE) = live-key count, values printed in tests/golden),
@@ -348,3 +348,27 @@ def tile_classes_brute(evict_at, block=BLOCK):
 def live_counts(evict_at):
     """n_i = number of keys visible to query i (one trace)."""
     return allowed(evict_at).sum(axis=1)
+
+
+# --------------------------------------------------------------------------
+# compaction event log -> evict_at
+# --------------------------------------------------------------------------
+def evict_at_from_events(cu_seqlens, events):
+    """events: rows (trace, when, start, end): at step ``when`` of trace ``trace`` the keys
+    [start, end) (trace-local) leave the cache (Sec. 2: the delete operator removes a span).
+    Key by key: evict_at[j] = the earliest ``when`` among the events whose span holds j,
+    2^31-1 if none.  Spans are clipped to the trace; rows naming no trace are ignored."""
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    total = int(cu[-1])
+    out = np.full(total, INF, dtype=np.int64)
+    ev = np.asarray(events, dtype=np.int64).reshape(-1, 4)
+    for b in range(len(cu) - 1):
+        T = int(cu[b + 1] - cu[b])
+        mine = ev[ev[:, 0] == b]
+        for j in range(T):
+            best = INF
+            for (_, when, a, z) in mine:
+                if a <= j < z and when < best:
+                    best = int(when)
+            out[cu[b] + j] = best
+    return out.astype(np.int32)

@@ -34,6 +34,7 @@ _vp, _i, _f, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_
 SIGNATURES = {
     "kvs_strerror": (ctypes.c_char_p, [_i]),
     "kvs_mask_meta_bytes": (_sz, [_i, _i, _i]),
+    "kvs_evict_at_from_events": (_i, [_vp, _i, _vp, _i, _i, _vp, _vp]),
     "kvs_mask_meta": (_i, [_vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "kvs_mask_meta_export": (_i, [_vp, _i, _vp, _i, _i, _vp, _vp, _vp, _vp]),
     "kvs_attn_fwd": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp]),
@@ -104,6 +105,19 @@ def _dev(t: torch.Tensor, name: str, dtype=None) -> int:
 # ------------------------------------------------------------------------------------------
 def kvs_mask_meta_bytes(batch: int, total_tokens: int, max_seqlen: int) -> int:
     return int(load().kvs_mask_meta_bytes(batch, total_tokens, max_seqlen))
+
+
+def kvs_evict_at_from_events(events: torch.Tensor, cu_seqlens: torch.Tensor, total_tokens: int,
+                             evict_at: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """events int32 [n, 4] rows (trace, when, start, end), cu_seqlens int32 [batch+1] (device).
+    Returns evict_at int32 [total_tokens]."""
+    if evict_at is None:
+        evict_at = torch.empty(total_tokens, dtype=torch.int32, device=cu_seqlens.device)
+    n = events.shape[0] if events.numel() else 0
+    _check(load().kvs_evict_at_from_events(_dev(events, "events", torch.int32) if n else None, n,
+                                           _dev(cu_seqlens, "cu_seqlens", torch.int32), cu_seqlens.numel() - 1, total_tokens,
+                                           _dev(evict_at, "evict_at", torch.int32), _stream(stream)), "kvs_evict_at_from_events")
+    return evict_at
 
 
 def kvs_mask_meta(evict_at: torch.Tensor, cu_seqlens: torch.Tensor, max_seqlen: int,

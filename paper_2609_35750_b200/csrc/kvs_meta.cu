@@ -197,9 +197,39 @@ meta_order_kernel(MetaHeader* hdr, const int32_t* __restrict__ blk_off, const in
     }
 }
 
+// ---- compaction event log -> evict_at ---------------------------------------------------------
+__global__ void evict_fill_kernel(int32_t* evict_at, int total_tokens) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < total_tokens) evict_at[i] = INT32_MAX;
+}
+
+// one CTA per event: the earliest `when` wins for every key of the span
+__global__ void evict_events_kernel(const int32_t* __restrict__ events, int n_events, const int32_t* __restrict__ cu_seqlens,
+                                    int batch, int32_t* evict_at) {
+    const int e = blockIdx.x;
+    if (e >= n_events) return;
+    const int b = events[4 * e + 0], when = events[4 * e + 1];
+    if (b < 0 || b >= batch) return;
+    const int tok0 = cu_seqlens[b];
+    const int T = cu_seqlens[b + 1] - tok0;
+    const int a = max(events[4 * e + 2], 0), z = min(events[4 * e + 3], T);
+    for (int j = a + threadIdx.x; j < z; j += blockDim.x) atomicMin(&evict_at[tok0 + j], when);
+}
+
 }  // namespace kvs
 
 using namespace kvs;
+
+extern "C" int kvs_evict_at_from_events(const int32_t* events, int n_events, const int32_t* cu_seqlens, int batch, int total_tokens,
+                                        int32_t* evict_at, kvs_stream_t stream) {
+    if (n_events < 0 || batch < 0 || total_tokens < 0) return KVS_ERR_INVALID_ARG;
+    if (total_tokens == 0) return KVS_OK;
+    if (!evict_at || !cu_seqlens || (n_events > 0 && !events)) return KVS_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    evict_fill_kernel<<<(total_tokens + 255) / 256, 256, 0, st>>>(evict_at, total_tokens);
+    if (n_events > 0) evict_events_kernel<<<n_events, 256, 0, st>>>(events, n_events, cu_seqlens, batch, evict_at);
+    return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
+}
 
 extern "C" size_t kvs_mask_meta_bytes(int batch, int total_tokens, int max_seqlen) {
     if (batch < 0 || total_tokens < 0 || max_seqlen < 0) return 0;

@@ -115,6 +115,82 @@ def fine_grained_evict_at(T: int, prompt: int, rng: np.random.Generator,
     return ev
 
 
+def events_to_evict_at(T: int, events) -> np.ndarray:
+    """Turns a compaction event log into ``evict_at``.  ``events`` is an iterable of
+    ``(when, start, end)``: at step ``when`` (the index of the first token generated after
+    the compaction) the keys ``[start, end)`` leave the cache.  A key named by several
+    events leaves at the earliest one."""
+    ev = np.full(T, INF, dtype=np.int32)
+    for when, a, b in events:
+        a, b = max(0, int(a)), min(T, int(b))
+        if b > a:
+            ev[a:b] = np.minimum(ev[a:b], np.int32(when))
+    return ev
+
+
+def _turn_bounds(T: int, prompt: int, turn_lens):
+    starts, ends = [], []
+    pos = min(prompt, T)
+    for L in turn_lens:
+        if pos >= T:
+            break
+        e = min(pos + int(L), T)
+        starts.append(pos)
+        ends.append(e)
+        pos = e
+    assert pos >= T, "turn_lens too short to fill the trace"
+    return starts, ends
+
+
+def markovian_thinker_events(T: int, prompt: int, turn_lens, budget: int):
+    """Markovian Thinker (Sec. 3: o = B/2, s = 0): whenever the live context (prompt excluded)
+    reaches ``budget`` tokens at the end of a turn, the oldest live turns are deleted until at
+    most half the budget remains.  Whole turns only (App. A.4).  Returns the event list."""
+    starts, ends = _turn_bounds(T, prompt, turn_lens)
+    live = []                       # indices of live turns, oldest first
+    events = []
+    for t in range(len(starts)):
+        live.append(t)
+        size = sum(ends[u] - starts[u] for u in live)
+        if size >= budget and ends[t] < T:
+            while live and size > budget // 2:
+                u = live.pop(0)
+                size -= ends[u] - starts[u]
+                events.append((ends[t], starts[u], ends[u]))
+    return events
+
+
+def markovian_pick_events(T: int, prompt: int, turn_lens, interval: int, keep: int, rng: np.random.Generator):
+    """Markovian Pick (Sec. 3): every ``interval`` turns the model chooses ``keep`` of the live
+    turns to retain and deletes all the others; here the choice is uniform at random, which
+    gives the arbitrary, non-contiguous retention the strategy allows."""
+    starts, ends = _turn_bounds(T, prompt, turn_lens)
+    live = []
+    events = []
+    for t in range(len(starts)):
+        live.append(t)
+        if (t + 1) % interval == 0 and ends[t] < T and len(live) > keep:
+            kept = set(rng.choice(len(live), size=keep, replace=False).tolist())
+            for idx, u in enumerate(live):
+                if idx not in kept:
+                    events.append((ends[t], starts[u], ends[u]))
+            live = [u for idx, u in enumerate(live) if idx in kept]
+    return events
+
+
+def single_evicted_turn_events(T: int, start: int, end: int, when: int):
+    """The controlled-retrieval mask (App. C.1 "Eviction and retrieval"): one early turn (the
+    assignment) leaves the cache before the answer tokens; everything else stays."""
+    return [(when, start, end)]
+
+
+def half_context_truncation_events(T: int, prompt: int):
+    """The SFT study's truncation mask (Sec. 6.1: half of the context masked, B = N/2): the
+    first half of the non-prompt context leaves once it has been generated."""
+    half = prompt + (T - prompt) // 2
+    return [(half, prompt, half)] if half > prompt else []
+
+
 # --------------------------------------------------------------------------
 # workloads
 # --------------------------------------------------------------------------
@@ -130,6 +206,7 @@ class Workload:
     softmax_scale: float = 0.0      # 0 => 1/sqrt(d)
     notes: str = ""
     rules: List[str] = field(default_factory=list)
+    events: Optional[np.ndarray] = None   # int32 [n, 4] rows (trace, when, start, end), when the mask came from an event log
 
     @property
     def batch(self) -> int:
@@ -237,7 +314,38 @@ def make_workload(cfg: int, seed: int = 0, shrink: int = 1,
         cu, eva = _pack([ev] * (batch or 1))
         return Workload(name, cu, eva, Hq or 64, Hkv or 8, 128,
                         notes="1 trace T=131072, prompt 1024, alternate keys evicted after 1+Geom(8192)")
+    if cfg in (5, 6, 7):
+        # further mask families through the same kernels (not in the five headline configs)
+        T, prompt = 65536 // s, 4096 // s
+        lo, hi = max(1, 256 // s), max(1, 2048 // s)
+        traces, log = [], []
+        for b in range(batch or 2):
+            r = _rng(seed, cfg, b)
+            lens = r.integers(lo, hi + 1, size=(T - prompt) // lo + 2)
+            if cfg == 5:
+                evs = markovian_thinker_events(T, prompt, lens, 16384 // s)
+            elif cfg == 6:
+                evs = markovian_pick_events(T, prompt, lens, 10, 4, r)
+            else:
+                evs = half_context_truncation_events(T, prompt) if b % 2 else \
+                    [(e, a, z) for (e, a, z) in _sliding_window_events(T, prompt, lens, 10)]
+            traces.append(events_to_evict_at(T, evs))
+            log += [(b, int(e), int(a), int(z)) for (e, a, z) in evs]
+        cu, eva = _pack(traces)
+        name = {5: "cfg5_markovian_thinker", 6: "cfg6_markovian_pick", 7: "cfg7_sft_random_masks"}[cfg]
+        note = {5: "turns U[256,2048], budget 16384: oldest turns deleted down to half the budget",
+                6: "turns U[256,2048], every 10 turns keep 4 random live turns",
+                7: "sliding window of 10 turns (stride 1) or half-context truncation, alternating"}[cfg]
+        return Workload(name, cu, eva, Hq or 32, Hkv or 8, 128, notes=f"{batch or 2} traces T={T}, prompt {prompt}; " + note,
+                        events=np.asarray(log, dtype=np.int32).reshape(-1, 4))
     raise ValueError(f"unknown config {cfg}")
+
+
+def _sliding_window_events(T: int, prompt: int, turn_lens, window: int):
+    """Sliding window over turns with stride 1 (Sec. 6.1: B = 10): when turn t ends, turn
+    t - window leaves."""
+    starts, ends = _turn_bounds(T, prompt, turn_lens)
+    return [(ends[t], starts[t - window], ends[t - window]) for t in range(window, len(starts))]
 
 
 # --------------------------------------------------------------------------

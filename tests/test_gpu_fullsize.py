@@ -31,6 +31,7 @@ CASES = [
     ("cfg3", dict(cfg=3)),
     ("cfg4", dict(cfg=4)),
     ("cfg4_control", dict(cfg=4, variant="control")),
+    ("cfg6_markovian_pick", dict(cfg=6)),          # non-monotone evict_at at full size
 ]
 
 

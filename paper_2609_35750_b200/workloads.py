@@ -192,6 +192,45 @@ def half_context_truncation_events(T: int, prompt: int):
 
 
 # --------------------------------------------------------------------------
+# re-prefill compaction: the comparison workload (Sec. 2 "Prefill-compaction", App. E)
+# --------------------------------------------------------------------------
+def reprefill_summary_lengths(T: int, prompt: int, work: int, summary: int) -> List[int]:
+    """Trace lengths when the Summary rollout of `summary_evict_at` is trained the re-prefill
+    way: every compaction starts a fresh trace that re-emits the retained entries (prompt and
+    the newest summary, r = prompt + summary) and then holds the next segment."""
+    lens, pos, first = [], min(prompt, T), True
+    while pos < T:
+        seg = min(work + summary, T - pos)
+        complete = seg == work + summary
+        lens.append((prompt if first else prompt + summary) + seg)
+        pos += seg
+        first = False
+        if not complete:
+            break
+    return lens
+
+
+def reprefill_keep_last_k_lengths(T: int, prompt: int, turn_lens, k: int) -> List[int]:
+    """Trace lengths when the keep-last-k-turns rollout is trained the re-prefill way: a
+    compaction happens at the end of every turn t >= k (turn t - k is deleted), and the fresh
+    trace re-emits the prompt and the k retained turns before generating the next turn."""
+    starts, ends = _turn_bounds(T, prompt, turn_lens)
+    n = len(starts)
+    if n <= k + 1:
+        return [T]
+    lens = [ends[k]]                                     # prompt + turns 0..k, no compaction yet
+    for u in range(k + 1, n):
+        retained = ends[u - 1] - starts[u - k]
+        lens.append(prompt + retained + (ends[u] - starts[u]))
+    return lens
+
+
+def reprefill_extra_entries(N: float, r: float, B: float) -> float:
+    """Closed form of the extra prefilled entries (Sec. 2): N r / (B - r)."""
+    return N * r / (B - r)
+
+
+# --------------------------------------------------------------------------
 # workloads
 # --------------------------------------------------------------------------
 @dataclass
@@ -251,6 +290,27 @@ def make_workload(cfg: int, seed: int = 0, shrink: int = 1,
     """
     s = int(shrink)
     assert s >= 1
+    if variant == "reprefill":
+        # the same rollouts cut into the fresh traces re-prefill compaction trains on: plain causal
+        # attention (nothing is evicted inside a trace), retained entries present again in every trace
+        if cfg == 1:
+            lens = reprefill_summary_lengths(32768 // s, 2048 // s, 4096 // s, 512 // s) * (batch or 4)
+            hq, hkv, pre, name = 28, 4, 1.0 / np.sqrt(128), "cfg1_reprefill"
+        elif cfg == 2:
+            T, prompt = 65536 // s, 4096 // s
+            lo, hi = max(1, 256 // s), max(1, 2048 // s)
+            lens = []
+            for b in range(batch or 2):
+                r = _rng(seed, 2, b)                       # the turn lengths of the KV-streams trace of config 2
+                tl = r.integers(lo, hi + 1, size=(T - prompt) // lo + 2)
+                lens += reprefill_keep_last_k_lengths(T, prompt, tl, 4)
+            hq, hkv, pre, name = 32, 8, 1.0, "cfg2_reprefill"
+        else:
+            raise ValueError("the re-prefill variant exists for configs 1 and 2")
+        cu = np.zeros(len(lens) + 1, dtype=np.int32)
+        cu[1:] = np.cumsum(lens)
+        return Workload(name, cu, np.full(int(cu[-1]), INF, dtype=np.int32), Hq or hq, Hkv or hkv, 128, q_prescale=pre,
+                        notes=f"{len(lens)} fresh traces, plain causal; retained entries re-emitted at every compaction")
     if cfg == 0:
         T, prompt, work, summ = 1024 // s, 128 // s, 192 // s, 32 // s
         ev = summary_evict_at(T, prompt, work, summ)

@@ -119,3 +119,41 @@ def test_retrieval_mask_parity_from_event_log_built_on_gpu():
     ev = B.kvs_evict_at_from_events(torch.from_numpy(events).cuda(), torch.from_numpy(cu).cuda(), T).cpu().numpy()
     w = W.Workload("retrieval", cu, ev, 4, 2, 128)
     _full_parity(w, seed=5)
+
+
+# ---- the re-prefill comparison workload (Sec. 2 "Prefill-compaction", App. E) ---------------------
+def test_reprefill_token_accounting_matches_the_closed_form():
+    # Summary layout of config 1: N = 30720 generated entries, r = prompt + summary = 2560 retained,
+    # b = 4608 new entries per compaction, budget B = r + b = 7168 (the peak live-key count)
+    lens = W.reprefill_summary_lengths(32768, 2048, 4096, 512)
+    assert lens == [6656, 7168, 7168, 7168, 7168, 7168, 5632] and max(lens) == 7168
+    extra = sum(lens) - 32768
+    assert extra == 6 * 2560                                  # six compactions, each re-emits r entries
+    closed = W.reprefill_extra_entries(30720, 2560, 7168)     # N r / (B - r), a continuous count of compactions
+    assert abs(closed - 30720 / 4608 * 2560) < 1e-9 and 0 <= closed - extra < 2560
+    # r = B/4 gives N/3 (the example printed with the derivation)
+    assert abs(W.reprefill_extra_entries(3000, 25, 100) - 1000) < 1e-9
+    # KV-streams prefills nothing again: the single trace has exactly N + prompt tokens
+    assert W.make_workload(1, batch=1).total_tokens == 32768
+    w = W.make_workload(1, variant="reprefill", batch=1)
+    assert w.total_tokens == sum(lens) and np.all(w.evict_at == W.INF)
+
+
+def test_reprefill_keep_last_k_by_hand_and_high_retention():
+    # prompt 2, turns 3,2,4,3 (T=14), keep 1: first trace = prompt + turns 0,1 = 7; then every turn u >= 2
+    # starts a trace with prompt + turn u-1 + turn u: 2+2+4 = 8, 2+4+3 = 9
+    assert W.reprefill_keep_last_k_lengths(14, 2, [3, 2, 4, 3], 1) == [7, 8, 9]
+    a, b = W.make_workload(2), W.make_workload(2, variant="reprefill")
+    ratio = b.total_tokens / a.total_tokens
+    # sliding window keeps almost the whole budget, so nearly everything is prefilled again at every turn:
+    # with r ~ prompt + 4 turns and b ~ one turn the closed form gives r / b ~ 7.6 extra copies
+    assert 6.0 < ratio < 9.0
+    mean_turn = (256 + 2048) / 2
+    closed = W.reprefill_extra_entries(65536 - 4096, 4096 + 4 * mean_turn, 4096 + 5 * mean_turn) / 65536
+    assert abs((ratio - 1.0) - closed) / closed < 0.15
+
+
+@pytest.mark.gpu
+def test_reprefill_workload_parity():
+    from tests.test_gpu_parity import _full_parity
+    _full_parity(W.make_workload(2, variant="reprefill", shrink=32, Hq=4, Hkv=2, batch=1), seed=3)

@@ -203,6 +203,50 @@ int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t* cu_seqlen
                           void* dq_host, void* dk_host, void* dv_host,
                           void* arena, size_t arena_bytes, kvs_stream_t stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * Rollout side (Sec. 1; Sec. 4 "Inference engine implementation"; App. A.3): the engine evicts KV
+ * entries directly in its paged cache and keeps decoding on the same stream.  Pages hold page_size
+ * tokens (16 in one engine, with turns padded to page multiples; 1 in the other):
+ *   k_cache, v_cache : bf16 [num_pages, page_size, Hkv, head_dim]
+ *   block_table      : int32 [num_seqs, max_pages], the pages of each sequence's LIVE cache, in order
+ *   n_tokens         : int32 [num_seqs], live tokens (every page full except possibly the last)
+ *   free_list        : int32 [4 + num_pages]: {top, status, -, -} then a stack of free page ids
+ * Eviction removes whole pages from a table and returns them to the stack; the rows never move.
+ * Decode attention reads exactly the pages a table names; it never sees a mask.  Device-side
+ * failures (cache full, a range that is not whole pages) set the status word, read with
+ * kvs_cache_status().
+ * ---------------------------------------------------------------------------------------------- */
+size_t kvs_cache_free_list_bytes(int num_pages);
+/* All pages free, status OK. */
+int kvs_cache_init(int32_t* free_list, int num_pages, kvs_stream_t stream);
+/* Appends one token (k_new, v_new: bf16 [num_seqs, Hkv, head_dim]) to every sequence whose `active`
+ * byte is non-zero (active == NULL: all), taking a page from the stack when the last one is full. */
+int kvs_cache_append(const void* k_new, const void* v_new, const uint8_t* active,
+                     int num_seqs, int Hkv, int head_dim, int page_size, int max_pages,
+                     int32_t* block_table, int32_t* n_tokens, int32_t* free_list,
+                     void* k_cache, void* v_cache, kvs_stream_t stream);
+/* Physical eviction.  ranges: int32 [n_ranges, 3] rows (sequence, first_page_slot, n_pages) in
+ * positions of the CURRENT table; the named table entries are removed (the rest keep their order),
+ * n_tokens drops by n_pages * page_size, the pages go back on the stack. */
+int kvs_cache_evict(const int32_t* ranges, int n_ranges, int num_seqs, int page_size, int max_pages,
+                    int32_t* block_table, int32_t* n_tokens, int32_t* free_list, kvs_stream_t stream);
+/* Reads the cache status word.  SYNCHRONISES the stream. */
+int kvs_cache_status(const int32_t* free_list, int* free_pages_host, kvs_stream_t stream);
+/* A split count that fills the GPU for this batch, and the workspace decode attention needs. */
+int kvs_decode_num_splits(int num_seqs, int Hkv, int max_tokens);
+size_t kvs_decode_workspace_bytes(int num_seqs, int Hq, int head_dim, int num_splits);
+/*
+ * One decode step: out[s,h] = softmax_j(scale * q[s,h].k_j) v_j over the live cache of sequence s
+ * (query head h reads KV head h / (Hq/Hkv)), lse[s,h] = log sum_j exp(scale * q.k_j).
+ * q, out: bf16 [num_seqs, Hq, head_dim]; lse: fp32 [num_seqs, Hq].  Hq/Hkv in {1,2,4,7,8}.
+ * A sequence with no live token gets out = 0, lse = -inf.
+ */
+int kvs_decode_attn(const void* q, const void* k_cache, const void* v_cache,
+                    const int32_t* block_table, const int32_t* n_tokens,
+                    int num_seqs, int Hq, int Hkv, int head_dim, int page_size, int max_pages,
+                    float softmax_scale, int num_splits, void* out, float* lse,
+                    void* workspace, size_t workspace_bytes, kvs_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -372,3 +372,44 @@ def evict_at_from_events(cu_seqlens, events):
                     best = int(when)
             out[cu[b] + j] = best
     return out.astype(np.int32)
+
+
+# --------------------------------------------------------------------------
+# paged KV cache with physical eviction (the engine's bookkeeping, Sec. 4 / App. A.3)
+# --------------------------------------------------------------------------
+class PagedCacheModel:
+    """Plain-Python model of the block tables and the free stack: pages of `page_size`
+    tokens; a sequence's table lists the pages of its live cache in order; eviction removes
+    table entries (whole pages) and pushes the pages back; appending pops a page when the
+    last one is full.  Page 0 is handed out first; freed pages are pushed in table order."""
+
+    def __init__(self, num_pages, page_size, num_seqs):
+        self.page_size = page_size
+        self.free = list(range(num_pages - 1, -1, -1))     # stack, top at the end
+        self.tables = [[] for _ in range(num_seqs)]
+        self.n_tokens = [0] * num_seqs
+
+    def append(self, s):
+        if self.n_tokens[s] % self.page_size == 0:
+            if not self.free:
+                raise RuntimeError("cache full")
+            self.tables[s].append(self.free.pop())
+        slot = self.n_tokens[s]
+        self.n_tokens[s] += 1
+        return self.tables[s][slot // self.page_size], slot % self.page_size
+
+    def evict(self, s, ranges):
+        """ranges: (first_page_slot, n_pages) in positions of the current table."""
+        npages = len(self.tables[s])
+        gone = set()
+        for a, cnt in ranges:
+            if a < 0 or cnt < 0 or a + cnt > npages:
+                raise ValueError("range outside the table")
+            if a + cnt == npages and cnt > 0 and self.n_tokens[s] % self.page_size != 0:
+                raise ValueError("the partially filled last page cannot leave")
+            gone.update(range(a, a + cnt))
+        kept = [p for i, p in enumerate(self.tables[s]) if i not in gone]
+        freed = [p for i, p in enumerate(self.tables[s]) if i in gone]
+        self.tables[s] = kept
+        self.free.extend(freed)
+        self.n_tokens[s] -= len(freed) * self.page_size

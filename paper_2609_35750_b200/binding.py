@@ -45,6 +45,14 @@ SIGNATURES = {
     "kvs_attn_bwd_noalloc": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp,
                                   ctypes.POINTER(ctypes.c_void_p), _vp]),
     "kvs_device_status": (_i, [_vp, _vp]),
+    "kvs_cache_free_list_bytes": (_sz, [_i]),
+    "kvs_cache_init": (_i, [_vp, _i, _vp]),
+    "kvs_cache_append": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "kvs_cache_evict": (_i, [_vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
+    "kvs_cache_status": (_i, [_vp, ctypes.POINTER(ctypes.c_int), _vp]),
+    "kvs_decode_num_splits": (_i, [_i, _i, _i]),
+    "kvs_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
+    "kvs_decode_attn": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _sz, _vp]),
     "kvs_host_arena_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "kvs_attn_fwd_bwd_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i,
                                    _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -259,3 +267,61 @@ def kvs_attn_fwd_bwd_host(evict_at, cu_seqlens, q, k, v, dout, max_seqlen: int, 
                                         out.data_ptr(), lse.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(),
                                         _dev(arena, "arena", torch.uint8), arena.numel(), _stream(stream)),
            "kvs_attn_fwd_bwd_host")
+
+
+# ------------------------------------------------------------------------------------------
+# rollout side: paged KV cache with physical eviction, decode attention
+# ------------------------------------------------------------------------------------------
+class PagedCache:
+    """Device buffers of a paged KV cache plus the calls that maintain it.  Holds no logic:
+    every operation is one call into the library."""
+
+    def __init__(self, num_pages: int, page_size: int, num_seqs: int, max_pages: int, Hkv: int, head_dim: int, device="cuda"):
+        self.num_pages, self.page_size, self.num_seqs, self.max_pages = num_pages, page_size, num_seqs, max_pages
+        self.Hkv, self.d = Hkv, head_dim
+        self.k_cache = torch.zeros((num_pages, page_size, Hkv, head_dim), dtype=torch.bfloat16, device=device)
+        self.v_cache = torch.zeros_like(self.k_cache)
+        self.block_table = torch.zeros((num_seqs, max_pages), dtype=torch.int32, device=device)
+        self.n_tokens = torch.zeros(num_seqs, dtype=torch.int32, device=device)
+        self.free_list = torch.zeros(int(load().kvs_cache_free_list_bytes(num_pages)) // 4, dtype=torch.int32, device=device)
+        _check(load().kvs_cache_init(self.free_list.data_ptr(), num_pages, _stream(None)), "kvs_cache_init")
+
+    def append(self, k_new: torch.Tensor, v_new: torch.Tensor, active: Optional[torch.Tensor] = None, stream=None) -> None:
+        _check(load().kvs_cache_append(_dev(k_new, "k_new", torch.bfloat16), _dev(v_new, "v_new", torch.bfloat16),
+                                       _dev(active, "active", torch.uint8) if active is not None else None,
+                                       self.num_seqs, self.Hkv, self.d, self.page_size, self.max_pages,
+                                       self.block_table.data_ptr(), self.n_tokens.data_ptr(), self.free_list.data_ptr(),
+                                       self.k_cache.data_ptr(), self.v_cache.data_ptr(), _stream(stream)), "kvs_cache_append")
+
+    def evict(self, ranges: torch.Tensor, stream=None) -> None:
+        """ranges int32 [n, 3] rows (sequence, first_page_slot, n_pages) (device)."""
+        n = ranges.shape[0] if ranges.numel() else 0
+        _check(load().kvs_cache_evict(_dev(ranges, "ranges", torch.int32) if n else None, n, self.num_seqs, self.page_size,
+                                      self.max_pages, self.block_table.data_ptr(), self.n_tokens.data_ptr(),
+                                      self.free_list.data_ptr(), _stream(stream)), "kvs_cache_evict")
+
+    def status(self, stream=None) -> Tuple[int, int]:
+        """(status code, free pages).  Synchronises."""
+        free = ctypes.c_int(0)
+        rc = int(load().kvs_cache_status(self.free_list.data_ptr(), ctypes.byref(free), _stream(stream)))
+        return rc, int(free.value)
+
+    def decode(self, q: torch.Tensor, softmax_scale: float = 0.0, num_splits: int = 0, out=None, lse=None, workspace=None,
+               max_tokens: Optional[int] = None, stream=None):
+        """q bf16 [num_seqs, Hq, d] -> (out bf16 [num_seqs, Hq, d], lse fp32 [num_seqs, Hq])."""
+        S, Hq, d = q.shape
+        if num_splits <= 0:
+            num_splits = int(load().kvs_decode_num_splits(S, self.Hkv, max_tokens or self.max_pages * self.page_size))
+        need = int(load().kvs_decode_workspace_bytes(S, Hq, d, num_splits))
+        if workspace is None:
+            workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+        if out is None:
+            out = torch.empty_like(q)
+        if lse is None:
+            lse = torch.empty((S, Hq), dtype=torch.float32, device=q.device)
+        _check(load().kvs_decode_attn(_dev(q, "q", torch.bfloat16), self.k_cache.data_ptr(), self.v_cache.data_ptr(),
+                                      self.block_table.data_ptr(), self.n_tokens.data_ptr(), S, Hq, self.Hkv, d, self.page_size,
+                                      self.max_pages, float(softmax_scale), num_splits, _dev(out, "out", torch.bfloat16),
+                                      _dev(lse, "lse", torch.float32), _dev(workspace, "workspace", torch.uint8),
+                                      workspace.numel(), _stream(stream)), "kvs_decode_attn")
+        return out, lse

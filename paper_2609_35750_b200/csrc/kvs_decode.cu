@@ -18,7 +18,6 @@
 namespace kvs {
 
 constexpr int DEC_THREADS = 128;
-constexpr int DEC_BLOCK = 16;        // tokens per softmax update
 
 struct DecodeParams {
     const __nv_bfloat16* q;          // [S, Hq, D]
@@ -32,31 +31,53 @@ struct DecodeParams {
     float* part_ml;                  // [S, Hq, nsplit, 2]  (max in base-2 units, sum)
 };
 
+// 16 bytes (CH = 8) or 8 bytes (CH = 4) of a bf16 row, widened to fp32
+template <int CH>
+struct RowChunk {
+    uint32_t w[CH / 2];
+    __device__ __forceinline__ void load(const __nv_bfloat16* ptr) {
+        if constexpr (CH == 8) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(ptr);
+            w[0] = raw.x; w[1] = raw.y; w[2] = raw.z; w[3] = raw.w;
+        } else {
+            const uint2 raw = *reinterpret_cast<const uint2*>(ptr);
+            w[0] = raw.x; w[1] = raw.y;
+        }
+    }
+    __device__ __forceinline__ void widen(float (&f)[CH]) const {
+#pragma unroll
+        for (int e = 0; e < CH / 2; ++e) {
+            f[2 * e] = __uint_as_float(w[e] << 16);               // low half: element 2e
+            f[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);   // high half: element 2e+1
+        }
+    }
+};
+
 template <int D, int G>
-__global__ void __launch_bounds__(DEC_THREADS)
+__global__ void __launch_bounds__(DEC_THREADS, (G > 4) ? 2 : 3)
 decode_partial_kernel(DecodeParams p) {
     constexpr int CH = D / 16;                  // elements of a row per lane (16 lanes per row): 8 or 4
+    constexpr int ROWS = (G > 4) ? 4 : 8;       // rows per half-warp per block (register budget)
+    constexpr int BLK = 2 * ROWS;               // tokens per softmax update
     const int z = blockIdx.x, g = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int half = lane >> 4, l16 = lane & 15;
     const int n = p.n_tokens[s];
     const int ps = p.page_size;
-    const int nblocks = (n + DEC_BLOCK - 1) / DEC_BLOCK;
+    const int nblocks = (n + BLK - 1) / BLK;
     // blocks of this split, dealt round-robin to (split, warp)
     const int stride = p.nsplit * (DEC_THREADS / 32);
     const int first = z * (DEC_THREADS / 32) + warp;
 
-    // q of the G heads: this lane's CH elements of each head, in fp32
+    // q of the G heads: this lane's CH elements of each head, in fp32, pre-scaled
     float qv[G][CH];
 #pragma unroll
     for (int h = 0; h < G; ++h) {
-        const __nv_bfloat16* qp = p.q + ((size_t)s * p.Hq + g * G + h) * D + l16 * CH;
+        RowChunk<CH> c;
+        c.load(p.q + ((size_t)s * p.Hq + g * G + h) * D + l16 * CH);
+        c.widen(qv[h]);
 #pragma unroll
-        for (int e = 0; e < CH; e += 2) {
-            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(qp + e));
-            qv[h][e] = f.x * p.scale_log2;
-            qv[h][e + 1] = f.y * p.scale_log2;
-        }
+        for (int e = 0; e < CH; ++e) qv[h][e] *= p.scale_log2;
     }
     float m_run[G], l_run[G], acc[G][CH];
 #pragma unroll
@@ -68,59 +89,61 @@ decode_partial_kernel(DecodeParams p) {
     }
     const int32_t* bt = p.block_table + (size_t)s * p.max_pages;
     const size_t row_stride = (size_t)p.Hkv * D;             // elements between tokens of a page
+    const size_t lane_off = (size_t)g * D + l16 * CH;
 
     for (int b = first; b < nblocks; b += stride) {
-        const int t0 = b * DEC_BLOCK;
-        // ---- scores of 16 tokens: this half-warp takes tokens t0 + 2r + half ----
-        float sc[DEC_BLOCK / 2][G];
+        const int t0 = b * BLK;
+        // row index (page * page_size + offset) of token t0 + l16, fetched once per block by every lane;
+        // tokens past the end are clamped to the last one (their scores are discarded below)
+        const int tl = min(t0 + (l16 & (BLK - 1)), n - 1);
+        const int my_row = bt[tl / ps] * ps + tl % ps;
+        // ---- all K rows of the block in flight, then the scores ----
+        RowChunk<CH> raw[ROWS];
+        int rowi[ROWS];
 #pragma unroll
-        for (int r = 0; r < DEC_BLOCK / 2; ++r) {
-            const int t = t0 + 2 * r + half;
-            float part[G];
+        for (int r = 0; r < ROWS; ++r) {
+            rowi[r] = __shfl_sync(0xffffffffu, my_row, 2 * r + half);
+            raw[r].load(p.k_cache + (size_t)rowi[r] * row_stride + lane_off);
+        }
+        float sc[ROWS][G];
 #pragma unroll
-            for (int h = 0; h < G; ++h) part[h] = 0.f;
-            if (t < n) {
-                const int page = bt[t / ps];
-                const __nv_bfloat16* kp = p.k_cache + ((size_t)page * ps + (t % ps)) * row_stride + (size_t)g * D + l16 * CH;
-                float kf[CH];
-                if constexpr (CH == 8) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(kp);
-                    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-                    const float2 b2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-                    const float2 c = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.z));
-                    const float2 d2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.w));
-                    kf[0] = a.x; kf[1] = a.y; kf[2] = b2.x; kf[3] = b2.y; kf[4] = c.x; kf[5] = c.y; kf[6] = d2.x; kf[7] = d2.y;
-                } else {
-                    const uint2 raw = *reinterpret_cast<const uint2*>(kp);
-                    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-                    const float2 b2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-                    kf[0] = a.x; kf[1] = a.y; kf[2] = b2.x; kf[3] = b2.y;
-                }
-#pragma unroll
-                for (int h = 0; h < G; ++h)
-#pragma unroll
-                    for (int e = 0; e < CH; ++e) part[h] = fmaf(qv[h][e], kf[e], part[h]);
-            }
+        for (int r = 0; r < ROWS; ++r) {
+            float kf[CH];
+            raw[r].widen(kf);
 #pragma unroll
             for (int h = 0; h < G; ++h) {
-                float v = part[h];
+                float v = 0.f;
 #pragma unroll
-                for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);      // within the 16 lanes of the row
-                sc[r][h] = (t < n) ? v : -INFINITY;
+                for (int e = 0; e < CH; ++e) v = fmaf(qv[h][e], kf[e], v);
+                sc[r][h] = v;
             }
         }
-        // ---- one softmax update per head for the 8 tokens of this half-warp ----
+        // ---- the V rows go in flight while the scores are reduced and exponentiated ----
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) raw[r].load(p.v_cache + (size_t)rowi[r] * row_stride + lane_off);
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) {
+            const bool ok = (t0 + 2 * r + half) < n;
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                float v = sc[r][h];
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);      // within the 16 lanes of the row
+                sc[r][h] = ok ? v : -INFINITY;
+            }
+        }
+        // one softmax update per head for the ROWS tokens of this half-warp
 #pragma unroll
         for (int h = 0; h < G; ++h) {
             float bm = sc[0][h];
 #pragma unroll
-            for (int r = 1; r < DEC_BLOCK / 2; ++r) bm = fmaxf(bm, sc[r][h]);
+            for (int r = 1; r < ROWS; ++r) bm = fmaxf(bm, sc[r][h]);
             const float m_new = fmaxf(m_run[h], bm);
             const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
             const float alpha = fast_exp2(m_run[h] - m_use);
             float sum = 0.f;
 #pragma unroll
-            for (int r = 0; r < DEC_BLOCK / 2; ++r) {
+            for (int r = 0; r < ROWS; ++r) {
                 sc[r][h] = fast_exp2(sc[r][h] - m_use);       // the score becomes the weight, in place
                 sum += sc[r][h];
             }
@@ -129,32 +152,15 @@ decode_partial_kernel(DecodeParams p) {
 #pragma unroll
             for (int e = 0; e < CH; ++e) acc[h][e] *= alpha;
         }
-        // ---- acc += p * v over the same tokens ----
+        // ---- acc += p * v (a token past the end has weight 0) ----
 #pragma unroll
-        for (int r = 0; r < DEC_BLOCK / 2; ++r) {
-            const int t = t0 + 2 * r + half;
-            if (t < n) {
-                const int page = bt[t / ps];
-                const __nv_bfloat16* vp = p.v_cache + ((size_t)page * ps + (t % ps)) * row_stride + (size_t)g * D + l16 * CH;
-                float vf[CH];
-                if constexpr (CH == 8) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(vp);
-                    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-                    const float2 b2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-                    const float2 c = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.z));
-                    const float2 d2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.w));
-                    vf[0] = a.x; vf[1] = a.y; vf[2] = b2.x; vf[3] = b2.y; vf[4] = c.x; vf[5] = c.y; vf[6] = d2.x; vf[7] = d2.y;
-                } else {
-                    const uint2 raw = *reinterpret_cast<const uint2*>(vp);
-                    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-                    const float2 b2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-                    vf[0] = a.x; vf[1] = a.y; vf[2] = b2.x; vf[3] = b2.y;
-                }
+        for (int r = 0; r < ROWS; ++r) {
+            float vf[CH];
+            raw[r].widen(vf);
 #pragma unroll
-                for (int h = 0; h < G; ++h)
+            for (int h = 0; h < G; ++h)
 #pragma unroll
-                    for (int e = 0; e < CH; ++e) acc[h][e] = fmaf(sc[r][h], vf[e], acc[h][e]);
-            }
+                for (int e = 0; e < CH; ++e) acc[h][e] = fmaf(sc[r][h], vf[e], acc[h][e]);
         }
     }
 
@@ -403,8 +409,9 @@ extern "C" int kvs_cache_evict(const int32_t* ranges, int n_ranges, int num_seqs
 
 extern "C" int kvs_decode_num_splits(int num_seqs, int Hkv, int max_tokens) {
     if (num_seqs <= 0 || Hkv <= 0 || max_tokens <= 0) return 1;
-    // enough CTAs for two waves on 148 SMs, but at least 4 blocks of 16 tokens per warp of a split
-    long long want = (2 * 148 + (long long)num_seqs * Hkv - 1) / ((long long)num_seqs * Hkv);
+    // enough CTAs for two waves at three resident CTAs per SM (148 SMs), but at least 4 blocks of 16
+    // tokens per warp of a split
+    long long want = (2 * 3 * 148 + (long long)num_seqs * Hkv - 1) / ((long long)num_seqs * Hkv);
     long long cap = ((long long)max_tokens + 16 * 4 * 4 - 1) / (16 * 4 * 4);
     long long n = want < cap ? want : cap;
     if (n < 1) n = 1;

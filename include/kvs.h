@@ -180,6 +180,17 @@ int kvs_attn_bwd_noalloc(const void* dout, const void* q, const void* k, const v
  */
 int kvs_device_status(const void* meta_or_workspace, kvs_stream_t stream);
 
+/*
+ * Self-test of the bounded device-side wait every kernel of the library uses (failure detection
+ * without a fault: no trap, no endless loop).  Launches one CTA whose threads wait on a barrier that
+ * needs `expected_arrivals` (1 or 2) arrivals while exactly one is made.  With 1 the wait completes and
+ * *status_word (device int32) stays KVS_OK; with 2 it can never complete: after limit_clocks SM clocks
+ * (at most 4e9) the first waiter records KVS_ERR_TIMEOUT there, all other waiters of the CTA fall
+ * through, and the kernel returns normally, leaving the context usable.
+ */
+int kvs_selftest_bounded_wait(int32_t* status_word, int expected_arrivals, long long limit_clocks,
+                              kvs_stream_t stream);
+
 /* Bytes of device arena needed by kvs_attn_fwd_bwd_host for these dims. */
 size_t kvs_host_arena_bytes(int batch, int total_tokens, int max_seqlen,
                             int Hq, int Hkv, int head_dim, int grad_dtype);

@@ -45,6 +45,7 @@ SIGNATURES = {
     "kvs_attn_bwd_noalloc": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp,
                                   ctypes.POINTER(ctypes.c_void_p), _vp]),
     "kvs_device_status": (_i, [_vp, _vp]),
+    "kvs_selftest_bounded_wait": (_i, [_vp, _i, ctypes.c_longlong, _vp]),
     "kvs_cache_free_list_bytes": (_sz, [_i]),
     "kvs_cache_init": (_i, [_vp, _i, _vp]),
     "kvs_cache_append": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -245,6 +246,14 @@ def kvs_device_status_ptr(device_address: int, stream=None) -> int:
 
 def kvs_device_status(buf: torch.Tensor, stream=None) -> int:
     return int(load().kvs_device_status(_dev(buf, "buf", torch.uint8), _stream(stream)))
+
+
+def kvs_selftest_bounded_wait(expected_arrivals: int, limit_clocks: int, stream=None) -> int:
+    """Runs the bounded-wait self-test and returns the status word (KVS_OK or KVS_ERR_TIMEOUT)."""
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(load().kvs_selftest_bounded_wait(word.data_ptr(), expected_arrivals, limit_clocks, _stream(stream)),
+           "kvs_selftest_bounded_wait")
+    return int(word.item())
 
 
 def kvs_host_arena_bytes(batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, grad_dtype) -> int:

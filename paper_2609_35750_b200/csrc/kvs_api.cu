@@ -89,6 +89,36 @@ extern "C" int kvs_device_status(const void* meta_or_workspace, kvs_stream_t str
     return h[1];
 }
 
+// ---- self-test of the bounded wait ---------------------------------------------------------------
+namespace kvs {
+// One CTA waits on an mbarrier that expects `expected` arrivals while only thread 0 arrives once:
+// with expected == 1 the wait completes; with expected == 2 nothing ever completes it, the wait gives
+// up after `limit_clocks`, records KVS_ERR_TIMEOUT, and every other waiter of the CTA falls through.
+__global__ void selftest_wait_kernel(int32_t* status, int expected, long long limit_clocks) {
+    __shared__ __align__(8) unsigned long long s_bar;
+    __shared__ int s_abort;
+    const uint32_t bar = smem_u32(&s_bar);
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        mbar_init(bar, (uint32_t)expected);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_arrive(bar);
+    mbar_wait_limit(bar, 0, &s_abort, status, limit_clocks);
+    __syncthreads();
+}
+}  // namespace kvs
+
+extern "C" int kvs_selftest_bounded_wait(int32_t* status_word, int expected_arrivals, long long limit_clocks, kvs_stream_t stream) {
+    if (!status_word || expected_arrivals < 1 || expected_arrivals > 2 || limit_clocks <= 0 || limit_clocks > 4000000000LL)
+        return KVS_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(status_word, 0, sizeof(int32_t), st) != cudaSuccess) return KVS_ERR_CUDA;
+    selftest_wait_kernel<<<1, 128, 0, st>>>(status_word, expected_arrivals, limit_clocks);
+    return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
+}
+
 // ---- whole path from host buffers ------------------------------------------------------------
 namespace {
 struct ArenaLayout {

@@ -175,18 +175,22 @@ __device__ __forceinline__ uint32_t mbar_try_wait_hint(uint32_t bar, uint32_t pa
 #ifndef KVS_WAIT_HINT_NS
 #define KVS_WAIT_HINT_NS 20000u
 #endif
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+__device__ __forceinline__ void mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                                long long limit_clocks) {
     if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
     while (true) {
         if (mbar_try_wait_hint(bar, parity, KVS_WAIT_HINT_NS)) return;
         if (*abort_flag) return;
-        if (clock64() - t0 > WAIT_LIMIT_CLOCKS) {
+        if (clock64() - t0 > limit_clocks) {
             *abort_flag = 1;
             set_status(status, KVS_ERR_TIMEOUT);
             return;
         }
     }
+}
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+    mbar_wait_limit(bar, parity, abort_flag, status, WAIT_LIMIT_CLOCKS);
 }
 
 // Register re-balancing between warp groups (all four warps of a warp group execute it).

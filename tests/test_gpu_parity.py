@@ -258,6 +258,19 @@ def test_bad_evict_at_is_reported_not_fatal():
     _full_parity(W.make_workload(0))
 
 
+def test_bounded_wait_gives_up_and_reports_without_hanging():
+    # failure detection without a fault: a wait that nothing can complete runs out after its limit, the kernel
+    # records KVS_ERR_TIMEOUT and returns; a wait that is completed reports nothing; the context stays usable
+    import time
+    assert B.kvs_selftest_bounded_wait(1, 200_000_000) == B.KVS_OK
+    t0 = time.time()
+    assert B.kvs_selftest_bounded_wait(2, 200_000_000) == B.KVS_ERR_TIMEOUT        # about 0.1 s of SM clocks
+    assert time.time() - t0 < 5.0
+    with pytest.raises(B.KvsError):
+        B.kvs_selftest_bounded_wait(3, 1000)
+    _full_parity(W.make_workload(0), bwd=False)
+
+
 def test_argument_errors():
     w = W.make_workload(0)
     q, k, v, do = (t.to(DEV) for t in W.make_tensors(w, 0))

@@ -250,8 +250,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 }
                 __syncwarp();
             }
-        } else if (warp == 13 && lane == 0) {
-            // ================= MMA issuer =================
+        } else if (warp == 13) {
+            // ================= MMA issuer (all lanes walk the loop, one elected lane issues) =================
+            const bool leader = elect_one();
             // descriptors of stage 0; a stage or a k-step adds a constant to the 14-bit address field
             const uint64_t dK_k = smem_desc(sK, 16, 1024), dV_k = smem_desc(sV, 16, 1024);
             const uint64_t dQ_k = smem_desc(sQ, 16, 1024), dDO_k = smem_desc(sDO, 16, 1024);
@@ -265,9 +266,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
                 const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
-                mma_ss(tmem_S, dK_k + off, dQ_k + off, IDESC_ST, kk > 0);
+                if (leader) mma_ss(tmem_S, dK_k + off, dQ_k + off, IDESC_ST, kk > 0);
             }
-            mma_commit(bar_s);
+            if (leader) mma_commit(bar_s);
             for (int j = 0; j < n_iter; ++j) {
                 const int s = j & 1;
                 const uint32_t ph = j & 1;
@@ -281,9 +282,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
-                    mma_ss(tmem_P, dV_k + off, dDO_k + off, IDESC_ST, kk > 0);
+                    if (leader) mma_ss(tmem_P, dV_k + off, dDO_k + off, IDESC_ST, kk > 0);
                 }
-                mma_commit(bar_dp);
+                if (leader) mma_commit(bar_dp);
                 KVS_TR(0, j, 4);
                 // dV(j) += P^T dO
                 mbar_wait(bar_p, ph, abort_flag, status);
@@ -291,9 +292,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 KVS_TR(0, j, 1);
 #pragma unroll
                 for (int kk = 0; kk < TILE / 16; ++kk)
-                    mma_ts(tmem_dV, tmem_S + (kk >> 2) * 64 + (kk & 3) * 8, dDO_mn + (uint64_t)(kk * 128), IDESC_KV,
+                    if (leader) mma_ts(tmem_dV, tmem_S + (kk >> 2) * 64 + (kk & 3) * 8, dDO_mn + (uint64_t)(kk * 128), IDESC_KV,
                            (j > 0) || (kk > 0));
-                mma_commit(bar_dofree);
+                if (leader) mma_commit(bar_dofree);
                 KVS_TR(0, j, 5);
                 // S^T(j+1) = K Q^T
                 if (j + 1 < n_iter) {
@@ -303,9 +304,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
                         const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
-                        mma_ss(tmem_S, dK_k + off, dQ_k + so1 + off, IDESC_ST, kk > 0);
+                        if (leader) mma_ss(tmem_S, dK_k + off, dQ_k + so1 + off, IDESC_ST, kk > 0);
                     }
-                    mma_commit(bar_s);
+                    if (leader) mma_commit(bar_s);
                 }
                 // dQ(j) = dS K, then dK(j) += dS^T Q.  Both read dS from shared memory: the same swizzled buffer
                 // is the MN-major A operand of dQ (queries contiguous) and, read as [keys x queries] rows, the
@@ -315,14 +316,14 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 KVS_TR(0, j, 6);
 #pragma unroll
                 for (int kk = 0; kk < TILE / 16; ++kk)
-                    mma_ss(tmem_P, dDS_mn + (uint64_t)(kk * 128), dK_mn + (uint64_t)(kk * 128), IDESC_DQ, kk > 0);
-                mma_commit(bar_dq);
+                    if (leader) mma_ss(tmem_P, dDS_mn + (uint64_t)(kk * 128), dK_mn + (uint64_t)(kk * 128), IDESC_DQ, kk > 0);
+                if (leader) mma_commit(bar_dq);
 #pragma unroll
                 for (int kk = 0; kk < TILE / 16; ++kk) {
                     const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
-                    mma_ss(tmem_dK, dDS_k + off, dQ_mn + so + (uint64_t)(kk * 128), IDESC_KV, (j > 0) || (kk > 0));
+                    if (leader) mma_ss(tmem_dK, dDS_k + off, dQ_mn + so + (uint64_t)(kk * 128), IDESC_KV, (j > 0) || (kk > 0));
                 }
-                mma_commit(bar_qfree(s));
+                if (leader) mma_commit(bar_qfree(s));
                 KVS_TR(0, j, 7);
             }
         }

@@ -5,12 +5,17 @@
 // query tiles.  384 threads in three warp groups:
 //   warps 0-3   softmax of tile 0 (one query row per thread)        } registers re-balanced with
 //   warps 4-7   softmax of tile 1                                    } setmaxnreg (208 / 208 / 88)
-//   warp 8      producer: TMA for Q0, Q1 and the K/V ring (2 stages); plain loads for evict_at
-//   warp 9      MMA issuer;  warps 10-11 idle
+//   warp 8      producer: TMA for Q0, Q1 and the K and V rings (2 stages each; K runs one key
+//               block ahead of V, its slot being released a whole iteration earlier); plain loads
+//               for evict_at
+//   warp 9      MMA issuer: all 32 lanes walk the loop and one elected lane issues, so descriptor
+//               arithmetic stays in uniform registers and an MMA costs a few issue slots even while
+//               the softmax warps of the same scheduler are busy;  warps 10-11 idle
 // Tensor memory: S0 [0,128)  S1 [128,256)  O0 [256,256+D)  O1 [384,384+D); P (bf16) overwrites S.
 // Per key block i the tensor pipe runs  O0 += P0 V, S0(i+1) = Q0 K^T, O1 += P1 V, S1(i+1) = Q1 K^T
 // while the two softmax groups alternate, so the exponentials of one tile overlap the MMAs of the
-// other.  EMPTY tiles are never visited (the CTA walks the row's non-empty list); the element mask
+// other.  A row's probabilities are handed over in two parts (the first P_SPLIT keys, then the
+// rest), so most of P V overlaps the last exponentials of the row.  EMPTY tiles are never visited (the CTA walks the row's non-empty list); the element mask
 // is evaluated on PARTIAL or ragged tiles only.  O is rescaled lazily: a row keeps its reference
 // maximum until the running maximum exceeds it by more than 8 (base-2), so exp2 arguments stay
 // below 2^8 and the rescale of O in tensor memory is rare.
@@ -20,6 +25,7 @@ namespace kvs {
 
 constexpr int FWD_THREADS = 384;
 constexpr float RESCALE_THRESHOLD = 8.0f;
+constexpr int P_SPLIT = 96;     // keys of a tile whose probabilities are handed to the MMA warp early
 
 template <int D>
 struct FwdSmem {
@@ -29,7 +35,7 @@ struct FwdSmem {
     static constexpr int OFF_EV = OFF_KV + 4 * TB;       // 2 stages x 128 int32
     static constexpr int OFF_FLAG = OFF_EV + 2 * TILE * 4;   // 2 stages x need_mask
     static constexpr int OFF_BAR = OFF_FLAG + 16;
-    static constexpr int OFF_MISC = OFF_BAR + 16 * 8;
+    static constexpr int OFF_MISC = OFF_BAR + 24 * 8;
     static constexpr int TOTAL = OFF_MISC + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024 + 1024;   // slack for the 1024-byte alignment (+ room for a debug trace)
 };
@@ -95,11 +101,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #endif
     const uint32_t bars = sbase + L::OFF_BAR;
     const uint32_t bar_q = bars;
-    auto bar_kvfull = [&](int s) { return bars + 8 * (1 + s); };    // TMA bytes of K and V
+    auto bar_vfull = [&](int s) { return bars + 8 * (1 + s); };     // TMA bytes of V
+    auto bar_kfull = [&](int s) { return bars + 8 * (16 + s); };    // TMA bytes of K
     auto bar_evfull = [&](int s) { return bars + 8 * (3 + s); };    // evict_at tile + need_mask flag (32 arrivals)
-    auto bar_kvfree = [&](int s) { return bars + 8 * (5 + s); };    // every MMA reading the stage has completed
+    auto bar_vfree = [&](int s) { return bars + 8 * (5 + s); };     // every P V product reading the stage's V has completed
+    auto bar_kfree = [&](int s) { return bars + 8 * (18 + s); };    // every Q K^T product reading the stage's K has completed
     auto bar_s = [&](int t) { return bars + 8 * (7 + t); };         // S_t ready
-    auto bar_p = [&](int t) { return bars + 8 * (9 + t); };         // P_t written (4 arrivals)
+    auto bar_p = [&](int t) { return bars + 8 * (9 + t); };         // all of P_t written (4 arrivals)
+    auto bar_p0 = [&](int t) { return bars + 8 * (14 + t); };       // first P_SPLIT keys of P_t written (4 arrivals)
     auto bar_evfree = [&](int s) { return bars + 8 * (11 + s); };   // softmax groups done with the evict_at tile
     const uint32_t bar_done = bars + 8 * 13;                         // all MMAs complete
 
@@ -107,12 +116,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         *abort_flag = 0;
         mbar_init(bar_q, 1);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(bar_kvfull(s), 1);
+            mbar_init(bar_vfull(s), 1);
+            mbar_init(bar_kfull(s), 1);
             mbar_init(bar_evfull(s), 32);
-            mbar_init(bar_kvfree(s), 1);
+            mbar_init(bar_vfree(s), 1);
+            mbar_init(bar_kfree(s), 1);
             mbar_init(bar_evfree(s), 4 * ntile);
             mbar_init(bar_s(s), 1);
             mbar_init(bar_p(s), 4);
+            mbar_init(bar_p0(s), 4);
         }
         mbar_init(bar_done, 1);
         fence_mbar_init();
@@ -135,19 +147,31 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 for (int t = 0; t < ntile; ++t)
                     for (int c = 0; c < NBOX; ++c) tma_load_3d(sQ + t * L::TB + c * BOX_BYTES, &tm_q, c * 64, h0 + t, tok0 + m * TILE, bar_q);
             }
+            // K runs one key block ahead of V: the slot of K(i+1) is released by the Q K^T products of
+            // block i-1, which are issued a whole iteration before the P V products that release V's slot.
+            auto load_k = [&](int i) {
+                const int s = i & 1;
+                if (i >= 2) mbar_wait(bar_kfree(s), ((i >> 1) + 1) & 1, abort_flag, status);
+                if (lane == 0) {
+                    mbar_expect_tx(bar_kfull(s), L::TB);
+                    const uint32_t dst = sKV + s * 2 * L::TB;
+                    for (int c = 0; c < NBOX; ++c) tma_load_3d(dst + c * BOX_BYTES, &tm_k, c * 64, g, tok0 + list[i] * TILE, bar_kfull(s));
+                }
+            };
+            if (nlist > 0) load_k(0);
             for (int i = 0; i < nlist; ++i) {
                 const int s = i & 1;
                 const int n = list[i];
                 if (i >= 2) {
-                    mbar_wait(bar_kvfree(s), ((i >> 1) + 1) & 1, abort_flag, status);
+                    mbar_wait(bar_vfree(s), ((i >> 1) + 1) & 1, abort_flag, status);
                     mbar_wait(bar_evfree(s), ((i >> 1) + 1) & 1, abort_flag, status);
                 }
                 if (lane == 0) {
-                    mbar_expect_tx(bar_kvfull(s), 2 * L::TB);
+                    mbar_expect_tx(bar_vfull(s), L::TB);
                     const uint32_t dst = sKV + s * 2 * L::TB;
-                    for (int c = 0; c < NBOX; ++c) tma_load_3d(dst + c * BOX_BYTES, &tm_k, c * 64, g, tok0 + n * TILE, bar_kvfull(s));
-                    for (int c = 0; c < NBOX; ++c) tma_load_3d(dst + L::TB + c * BOX_BYTES, &tm_v, c * 64, g, tok0 + n * TILE, bar_kvfull(s));
+                    for (int c = 0; c < NBOX; ++c) tma_load_3d(dst + L::TB + c * BOX_BYTES, &tm_v, c * 64, g, tok0 + n * TILE, bar_vfull(s));
                 }
+                if (i + 1 < nlist) load_k(i + 1);
                 const bool need_mask = (cls[n] != KVS_CLASS_FULL) || (n * TILE + TILE > T);
                 if (need_mask) {
 #pragma unroll
@@ -159,8 +183,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 if (lane == 0) sFlag[s] = need_mask ? 1 : 0;
                 mbar_arrive(bar_evfull(s));
             }
-        } else if (warp == 9 && lane == 0) {
-            // ================= MMA issuer =================
+        } else if (warp == 9) {
+            // ================= MMA issuer (all lanes walk the loop, one elected lane issues) =================
+            const bool leader = elect_one();
             const uint64_t dQ0 = smem_desc(sQ, 16, 1024);
             const uint64_t dK0 = smem_desc(sKV, 16, 1024);
             const uint64_t dV0 = smem_desc(sKV + L::TB, BOX_BYTES, 1024);
@@ -169,41 +194,55 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
-                    mma_ss(tmem + t * 128, dQ0 + t * TBU + off, dK0 + s * 2 * TBU + off, IDESC_S, kk > 0);
+                    if (leader) mma_ss(tmem + t * 128, dQ0 + t * TBU + off, dK0 + s * 2 * TBU + off, IDESC_S, kk > 0);
                 }
-                mma_commit(bar_s(t));
+                if (leader) mma_commit(bar_s(t));
             };
             if (nlist > 0) {
                 mbar_wait(bar_q, 0, abort_flag, status);
-                mbar_wait(bar_kvfull(0), 0, abort_flag, status);
+                mbar_wait(bar_kfull(0), 0, abort_flag, status);
                 tc_fence_after();
                 for (int t = 0; t < ntile; ++t) issue_s(t, 0);
+                if (leader) mma_commit(bar_kfree(0));
             }
             for (int i = 0; i < nlist; ++i) {
                 const int s = i & 1;
                 for (int t = 0; t < ntile; ++t) {
                     // O_t += P_t V(i):  A = P rows from tensor memory (16 keys = 8 packed columns per step),
                     //                   B = V, MN-major, 16 key rows per step
+                    // The first P_SPLIT keys of P arrive while the row's last exponentials are still being
+                    // taken, so most of this product overlaps the tail of the softmax.
                     KVS_TRF(i, t * 4 + 0);
-                    mbar_wait(bar_p(t), i & 1, abort_flag, status);
+                    mbar_wait(bar_p0(t), i & 1, abort_flag, status);
+                    if (t == 0) mbar_wait(bar_vfull(s), (i >> 1) & 1, abort_flag, status);
                     tc_fence_after();
                     KVS_TRF(i, t * 4 + 1);
 #pragma unroll
-                    for (int kk = 0; kk < TILE / 16; ++kk)
-                        mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, dV0 + s * 2 * TBU + (uint64_t)(kk * 128), IDESC_O,
+                    for (int kk = 0; kk < P_SPLIT / 16; ++kk)
+                        if (leader) mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, dV0 + s * 2 * TBU + (uint64_t)(kk * 128), IDESC_O,
                                (i > 0) || (kk > 0));
-                    if (t == ntile - 1) mma_commit(bar_kvfree(s));      // K(i), V(i) no longer read by anything issued later
+                    if (t == 0) KVS_TRF(i, 9);
+                    mbar_wait(bar_p(t), i & 1, abort_flag, status);
+                    tc_fence_after();
+                    if (t == 0) KVS_TRF(i, 10);
+#pragma unroll
+                    for (int kk = P_SPLIT / 16; kk < TILE / 16; ++kk)
+                        if (leader) mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, dV0 + s * 2 * TBU + (uint64_t)(kk * 128), IDESC_O, true);
+                    if (leader && t == ntile - 1) mma_commit(bar_vfree(s));       // V(i) is not read by anything issued later
                     if (i + 1 < nlist) {
+                        KVS_TRF(i, t * 4 + 3);
                         if (t == 0) {
-                            mbar_wait(bar_kvfull(s ^ 1), ((i + 1) >> 1) & 1, abort_flag, status);
+                            mbar_wait(bar_kfull(s ^ 1), ((i + 1) >> 1) & 1, abort_flag, status);
                             tc_fence_after();
+                            KVS_TRF(i, 15);
                         }
                         issue_s(t, s ^ 1);
+                        if (leader && t == ntile - 1) mma_commit(bar_kfree(s ^ 1));
                     }
                     KVS_TRF(i, t * 4 + 2);
                 }
             }
-            mma_commit(bar_done);
+            if (leader) mma_commit(bar_done);
         }
     } else {
         // ================= softmax groups =================
@@ -246,7 +285,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         sv[96 + e] = __uint_as_float(r3[e]);
                     }
                 }
-                if (tid == 0) KVS_TRF(i, 9);
+                
                 if (need_mask) {
                     const int4* ev4 = reinterpret_cast<const int4*>(sEv + s * TILE);
 #pragma unroll
@@ -261,17 +300,17 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_evfree(s));
-                // eight independent partial maxima, then a short tree (no 127-deep dependency chain)
+                // eight independent partial maxima (three-input max), then a short tree
                 float mx[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) mx[u] = sv[u];
+                for (int u = 0; u < 8; ++u) mx[u] = fmaxf(sv[u], sv[8 + u]);
 #pragma unroll
-                for (int e = 8; e < TILE; e += 8) {
+                for (int e = 16; e < TILE; e += 16) {
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) mx[u] = fmaxf(mx[u], sv[e + u]);
+                    for (int u = 0; u < 8; ++u) mx[u] = fmax3(mx[u], sv[e + u], sv[e + 8 + u]);
                 }
                 const float tile_max =
-                    fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
+                    fmaxf(fmax3(mx[0], mx[1], mx[2]), fmaxf(fmax3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
                 // lazy rescale: move the reference only when the maximum ran away from it
                 const bool grow = (tile_max > ref_max + RESCALE_THRESHOLD) || (ref_max == -INFINITY && tile_max > -INFINITY);
                 if (__any_sync(0xffffffffu, grow)) {
@@ -291,7 +330,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         }
                     }
                 }
-                if (tid == 0) KVS_TRF(i, 10);
                 const float neg_ref = (ref_max == -INFINITY) ? 0.f : -ref_max;
                 // packed fp32x2: one multiply-add forms two exponents, one add accumulates two terms
                 const float2 c2 = make_float2(p.scale_log2, p.scale_log2);
@@ -307,23 +345,37 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         ts[u] = __fadd2_rn(ts[u], pp);
                         pk[(e >> 1) + u] = pack_bf16(pp.x, pp.y);
                     }
+                    if (e + 8 == P_SPLIT) {
+                        // P (bf16, packed two per column) goes over the S columns already read; the first
+                        // P_SPLIT keys are handed to the MMA warp before the rest of the row is done
+                        uint32_t r[32], r2[16];
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) r[c] = pk[c];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) r2[c] = pk[32 + c];
+                        tmem_st32(tmem_S, r);
+                        tmem_st16(tmem_S + 32, r2);
+                        tmem_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_p0(t));
+                    }
                 }
                 const float2 t01 = __fadd2_rn(ts[0], ts[1]), t23 = __fadd2_rn(ts[2], ts[3]);
                 const float tile_sum = (t01.x + t01.y) + (t23.x + t23.y);
-                if (tid == 0) KVS_TRF(i, 11);
+                
                 run_sum += tile_sum;
+                {
+                    uint32_t r2[16];
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t r[32];
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) r[e] = pk[c * 32 + e];
-                    tmem_st32(tmem_S + c * 32, r);         // P (bf16, 64 columns) over the S columns already read
+                    for (int c = 0; c < 16; ++c) r2[c] = pk[48 + c];
+                    tmem_st16(tmem_S + 48, r2);
                 }
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p(t));
-                if (tid == 0) KVS_TRF(i, 12);
+                if (t == 0 && tid == 0) KVS_TRF(i, 12);
                 if (tid == 128) KVS_TRF(i, 14);
             }
 

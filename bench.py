@@ -29,7 +29,7 @@ METRIC = "masked_attn_fwd_bwd_effective_tflops"
 UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the backward main kernel, from the
 # ncu captures summarised under profiles/ (None until a capture of that workload exists)
-NCU_DRAM_BYTES_PER_LAUNCH = {"cfg2_keep_last_4_turns": 20469301248}   # profiles/bwd_kernel_cfg2.md, full-size light pass
+NCU_DRAM_BYTES_PER_LAUNCH = {"cfg2_keep_last_4_turns": 20461770496}   # profiles/bwd_kernel_cfg2.md, full-size light pass
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

@@ -25,9 +25,37 @@ def main():
     ap.add_argument("--hq", type=int, default=None)
     ap.add_argument("--hkv", type=int, default=None)
     ap.add_argument("--grad", type=str, default="bf16", choices=["bf16", "fp32"])
+    ap.add_argument("--batch", type=int, default=None, help="number of traces (default: the config's own)")
+    ap.add_argument("--meta-only", action="store_true",
+                    help="run only the mask-metadata pass (no q/k/v tensors): lets the batch be large enough for its bandwidth to show")
     a = ap.parse_args()
     dev = "cuda"
-    w = W.make_workload(a.config, seed=0, shrink=a.shrink, Hq=a.hq, Hkv=a.hkv, variant=a.variant)
+    w = W.make_workload(a.config, seed=0, shrink=a.shrink, Hq=a.hq, Hkv=a.hkv, variant=a.variant, batch=a.batch)
+    if a.meta_only:
+        ev = torch.from_numpy(w.evict_at).to(dev)
+        cu = torch.from_numpy(w.cu_seqlens).to(dev)
+        nbytes = B.kvs_mask_meta_bytes(w.batch, w.total_tokens, w.max_seqlen)
+        meta = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        ms = []
+        for _ in range(max(a.iters, 3)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.kvs_mask_meta(ev, cu, w.max_seqlen, meta_buf=meta)
+            e1.record()
+            torch.cuda.synchronize()
+            ms.append(e0.elapsed_time(e1))
+        st = B.kvs_device_status(meta)
+        nb = sum(-(-int(t) // 128) for t in (w.cu_seqlens[1:] - w.cu_seqlens[:-1]))
+        tiles = sum((-(-int(t) // 128)) ** 2 for t in (w.cu_seqlens[1:] - w.cu_seqlens[:-1]))
+        # algorithmic bytes: evict_at read once and copied once (4 + 4 B per token), one class byte and one
+        # 2-byte list slot per tile of the per-trace square
+        alg = 8 * w.total_tokens + 3 * tiles
+        print(json.dumps({"workload": w.name, "traces": w.batch, "tokens": w.total_tokens, "key_blocks": nb, "tiles": tiles,
+                          "meta_buffer_bytes": nbytes, "status": st, "ms": ms, "algorithmic_bytes": alg,
+                          "gbs_last": alg / (ms[-1] * 1e-3) / 1e9}))
+        if st != 0:
+            raise SystemExit(1)
+        return
     q, k, v, do = W.make_tensors(w, seed=0, device=dev)
     ev = torch.from_numpy(w.evict_at).to(dev)
     cu = torch.from_numpy(w.cu_seqlens).to(dev)

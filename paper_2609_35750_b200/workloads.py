@@ -19,6 +19,7 @@ Conventions
 """
 from __future__ import annotations
 
+import dataclasses
 from dataclasses import dataclass, field
 from typing import List, Optional
 
@@ -286,10 +287,16 @@ def make_workload(cfg: int, seed: int = 0, shrink: int = 1,
     layout (trace, prompt, segment, turn) by an integer so that the CPU oracle
     can run the whole tensor; head counts and batch may be overridden for the
     same reason.  ``variant``: cfg 1 "B" (scale folded into Q, softmax scale
-    1); cfg 4 "control" (no eviction) or "b" (every non-prompt key evicted).
+    1); cfg 4 "b" (every non-prompt key evicted); any cfg "control" (same
+    shapes and values, nothing ever evicted: plain causal attention);
+    cfg 1, 2 "reprefill" (the rollouts cut into re-prefill's fresh traces).
     """
     s = int(shrink)
     assert s >= 1
+    if variant == "control" and cfg != 4:
+        w = make_workload(cfg, seed, shrink, Hq, Hkv, batch, "")
+        return dataclasses.replace(w, name=w.name + "_control_causal", evict_at=np.full_like(w.evict_at, INF),
+                                   rules=None, events=None, notes=w.notes + "; control: evict_at = INF everywhere")
     if variant == "reprefill":
         # the same rollouts cut into the fresh traces re-prefill compaction trains on: plain causal
         # attention (nothing is evicted inside a trace), retained entries present again in every trace

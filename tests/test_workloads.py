@@ -123,3 +123,14 @@ def test_make_tensors_deterministic_and_bf16():
         assert x.dtype == torch.bfloat16 and torch.equal(x, y)
     assert not torch.equal(a[0], c[0])
     assert a[0].shape == (1024, 4, 64) and a[1].shape == (1024, 4, 64)
+
+
+def test_control_variant_of_any_config_is_plain_causal():
+    for cfg in (0, 2, 3):
+        a = W.make_workload(cfg, shrink=8 if cfg else 1)
+        c = W.make_workload(cfg, shrink=8 if cfg else 1, variant="control")
+        assert np.array_equal(a.cu_seqlens, c.cu_seqlens) and (a.Hq, a.Hkv, a.d) == (c.Hq, c.Hkv, c.d)
+        assert np.all(c.evict_at == W.INF) and c.name.endswith("_control_causal")
+        lens = np.diff(c.cu_seqlens).astype(np.int64)
+        assert W.count_pairs(c) == int((lens * (lens + 1) // 2).sum())      # closed form of the causal triangle
+        assert W.count_pairs(a) < W.count_pairs(c)

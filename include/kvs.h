@@ -201,9 +201,11 @@ size_t kvs_host_arena_bytes(int batch, int total_tokens, int max_seqlen,
  * backward, copies out, lse, dq, dk, dv back, and SYNCHRONISES the stream.  Host buffers
  * should be page-locked for the copies to be asynchronous.  arena: device memory the caller
  * provides, >= kvs_host_arena_bytes(...), 256-byte aligned.  Returns the device status.
- * The copy of dout overlaps the forward and the copies of out and lse overlap the backward, on an
- * internal stream that (with four events) is created and destroyed inside the call; no device memory
- * is allocated.
+ * The work is pipelined over the Hkv KV-head groups, which are independent: while one group's
+ * forward and backward run, the next group's inputs are uploaded and the previous group's results
+ * downloaded, on two internal streams that (with their events) are created and destroyed inside
+ * the call; no device memory is allocated.  The arena holds three groups at a time, so it is
+ * smaller than the tensors when Hkv > 3.
  */
 int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t* cu_seqlens_host,
                           const void* q_host, const void* k_host, const void* v_host,

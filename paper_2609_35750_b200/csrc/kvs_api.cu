@@ -2,6 +2,7 @@
 #include <cudaTypedefs.h>
 
 #include "kvs_common.cuh"
+#include <vector>
 
 namespace kvs {
 
@@ -120,42 +121,61 @@ extern "C" int kvs_selftest_bounded_wait(int32_t* status_word, int expected_arri
 }
 
 // ---- whole path from host buffers ------------------------------------------------------------
+// The work is cut into one chunk per KV head (its G query heads, all tokens): chunks are independent
+// in the forward and the backward, so while chunk c computes, the inputs of chunk c+1 arrive and
+// the results of chunk c-1 leave (PCIe is full duplex; two copy streams besides the caller's).
+// Each chunk lives in one of HOST_SLOTS sets of contiguous [tokens, G, d] / [tokens, 1, d] buffers,
+// packed and unpacked by strided 2-D copies; the kernels run on a chunk as on any (Hq = G, Hkv = 1) problem.
 namespace {
+constexpr int HOST_SLOTS = 3;
+// A slot's workspace status is reset by the next chunk that uses the slot; the first failure is kept here.
+__global__ void fold_status_kernel(const int32_t* ws_words, int32_t* sticky) {
+    if (ws_words[1] != KVS_OK && *sticky == KVS_OK) *sticky = ws_words[1];
+}
 struct ArenaLayout {
-    size_t evict, cu, q, k, v, dout, out, lse, dq, dk, dv, meta, ws, total;
-    size_t meta_bytes, ws_bytes, nq_bytes, nkv_bytes, gq_bytes, gkv_bytes, lse_bytes;
+    size_t evict, cu, sticky, meta, slot0, slot_stride, total;      // global part, then HOST_SLOTS equal slots
+    size_t q, k, v, dout, out, lse, dq, dk, dv, ws;          // offsets inside a slot
+    size_t meta_bytes, ws_bytes, nq_bytes, nkv_bytes, gq_bytes, gkv_bytes, lse_bytes;   // per chunk
+    int slots;
 };
 ArenaLayout arena_layout(int batch, int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim, int grad_dtype) {
     ArenaLayout A;
+    const int G = Hq / Hkv;
     const size_t gsz = grad_dtype == KVS_GRAD_FP32 ? 4 : 2;
-    A.nq_bytes = (size_t)total_tokens * Hq * head_dim * 2;
-    A.nkv_bytes = (size_t)total_tokens * Hkv * head_dim * 2;
-    A.gq_bytes = (size_t)total_tokens * Hq * head_dim * gsz;
-    A.gkv_bytes = (size_t)total_tokens * Hkv * head_dim * gsz;
-    A.lse_bytes = (size_t)total_tokens * Hq * 4;
+    A.slots = Hkv < HOST_SLOTS ? Hkv : HOST_SLOTS;
+    A.nq_bytes = (size_t)total_tokens * G * head_dim * 2;
+    A.nkv_bytes = (size_t)total_tokens * head_dim * 2;
+    A.gq_bytes = (size_t)total_tokens * G * head_dim * gsz;
+    A.gkv_bytes = (size_t)total_tokens * head_dim * gsz;
+    A.lse_bytes = (size_t)total_tokens * G * 4;
     A.meta_bytes = kvs_mask_meta_bytes(batch, total_tokens, max_seqlen);
-    A.ws_bytes = kvs_attn_bwd_workspace_bytes(total_tokens, Hq, Hkv, head_dim, grad_dtype);
+    A.ws_bytes = kvs_attn_bwd_workspace_bytes(total_tokens, G, 1, head_dim, grad_dtype);
     size_t o = 0;
     A.evict = o; o = align_up(o + (size_t)total_tokens * 4, 256);
     A.cu = o;    o = align_up(o + (size_t)(batch + 1) * 4, 256);
-    A.q = o;     o = align_up(o + A.nq_bytes, 256);
-    A.k = o;     o = align_up(o + A.nkv_bytes, 256);
-    A.v = o;     o = align_up(o + A.nkv_bytes, 256);
-    A.dout = o;  o = align_up(o + A.nq_bytes, 256);
-    A.out = o;   o = align_up(o + A.nq_bytes, 256);
-    A.lse = o;   o = align_up(o + A.lse_bytes, 256);
-    A.dq = o;    o = align_up(o + A.gq_bytes, 256);
-    A.dk = o;    o = align_up(o + A.gkv_bytes, 256);
-    A.dv = o;    o = align_up(o + A.gkv_bytes, 256);
+    A.sticky = o; o += 256;
     A.meta = o;  o = align_up(o + A.meta_bytes, 256);
-    A.ws = o;    o = align_up(o + A.ws_bytes, 256);
-    A.total = o;
+    A.slot0 = o;
+    size_t t = 0;
+    A.q = t;     t = align_up(t + A.nq_bytes, 256);
+    A.k = t;     t = align_up(t + A.nkv_bytes, 256);
+    A.v = t;     t = align_up(t + A.nkv_bytes, 256);
+    A.dout = t;  t = align_up(t + A.nq_bytes, 256);
+    A.out = t;   t = align_up(t + A.nq_bytes, 256);
+    A.lse = t;   t = align_up(t + A.lse_bytes, 256);
+    A.dq = t;    t = align_up(t + A.gq_bytes, 256);
+    A.dk = t;    t = align_up(t + A.gkv_bytes, 256);
+    A.dv = t;    t = align_up(t + A.gkv_bytes, 256);
+    A.ws = t;    t = align_up(t + A.ws_bytes, 256);
+    A.slot_stride = t;
+    A.total = A.slot0 + (size_t)A.slots * A.slot_stride;
     return A;
 }
 }  // namespace
 
 extern "C" size_t kvs_host_arena_bytes(int batch, int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim, int grad_dtype) {
     if (batch < 0 || total_tokens < 0 || max_seqlen < 0 || Hq <= 0 || Hkv <= 0 || head_dim <= 0) return 0;
+    if (Hq % Hkv != 0) return 0;
     if (grad_dtype != KVS_GRAD_BF16 && grad_dtype != KVS_GRAD_FP32) return 0;
     return arena_layout(batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, grad_dtype).total;
 }
@@ -167,7 +187,7 @@ extern "C" int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t
                                      size_t arena_bytes, kvs_stream_t stream) {
     if (batch < 0 || total_tokens < 0 || max_seqlen < 0 || Hq <= 0 || Hkv <= 0) return KVS_ERR_INVALID_ARG;
     if (head_dim != 64 && head_dim != 128) return KVS_ERR_UNSUPPORTED;
-    if (Hq % Hkv != 0) return KVS_ERR_UNSUPPORTED;
+    if (Hq % Hkv != 0 || Hkv > 1024) return KVS_ERR_UNSUPPORTED;
     if (grad_dtype != KVS_GRAD_BF16 && grad_dtype != KVS_GRAD_FP32) return KVS_ERR_INVALID_ARG;
     if (total_tokens == 0 || batch == 0) return KVS_OK;
     if (!evict_at_host || !cu_seqlens_host || !q_host || !k_host || !v_host || !dout_host || !out_host || !lse_host || !dq_host ||
@@ -178,67 +198,98 @@ extern "C" int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t
     if (arena_bytes < A.total) return KVS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     char* a = (char*)arena;
-    // A second stream carries the copies that can overlap compute (PCIe is full duplex): dout goes in
-    // while the forward runs, out and lse come back while the backward runs.  Stream and events live
-    // for this call only.
-    cudaStream_t cp = nullptr;
-    cudaEvent_t ev_in = nullptr, ev_fwd = nullptr, ev_dout = nullptr, ev_out = nullptr;
-    struct Cleanup {
-        cudaStream_t& cp;
-        cudaEvent_t &e0, &e1, &e2, &e3;
-        ~Cleanup() {
-            if (e0) cudaEventDestroy(e0);
-            if (e1) cudaEventDestroy(e1);
-            if (e2) cudaEventDestroy(e2);
-            if (e3) cudaEventDestroy(e3);
-            if (cp) cudaStreamDestroy(cp);
+    const int G = Hq / Hkv;
+    const int NC = Hkv;                                    // chunks
+    const size_t gsz = grad_dtype == KVS_GRAD_FP32 ? 4 : 2;
+    // Two copy streams and four events per chunk, all created and destroyed inside this call.
+    struct Res {
+        cudaStream_t in = nullptr, outs = nullptr;
+        std::vector<cudaEvent_t> ev;
+        ~Res() {
+            for (cudaEvent_t e : ev)
+                if (e) cudaEventDestroy(e);
+            if (in) cudaStreamDestroy(in);
+            if (outs) cudaStreamDestroy(outs);
         }
-    } cleanup{cp, ev_in, ev_fwd, ev_dout, ev_out};
-    if (cudaStreamCreateWithFlags(&cp, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
-    if (cudaEventCreateWithFlags(&ev_in, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ev_fwd, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ev_dout, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ev_out, cudaEventDisableTiming) != cudaSuccess)
-        return KVS_ERR_CUDA;
-#define KVS_CP(strm, dst, src, bytes, kind) \
-    if (cudaMemcpyAsync(dst, src, bytes, kind, strm) != cudaSuccess) return KVS_ERR_CUDA
+    } R;
+    if (cudaStreamCreateWithFlags(&R.in, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
+    if (cudaStreamCreateWithFlags(&R.outs, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
+    R.ev.assign((size_t)NC * 5 + 1, nullptr);
+    for (cudaEvent_t& e : R.ev)
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return KVS_ERR_CUDA;
+    auto ev_qkv = [&](int c) { return R.ev[(size_t)c * 5 + 0]; };    // q, k, v of chunk c are on the device
+    auto ev_dout = [&](int c) { return R.ev[(size_t)c * 5 + 1]; };   // dout of chunk c is on the device
+    auto ev_fwd = [&](int c) { return R.ev[(size_t)c * 5 + 2]; };    // forward of chunk c done
+    auto ev_bwd = [&](int c) { return R.ev[(size_t)c * 5 + 3]; };    // backward of chunk c done
+    auto ev_down = [&](int c) { return R.ev[(size_t)c * 5 + 4]; };   // every result of chunk c is on the host
+    cudaEvent_t ev_start = R.ev[(size_t)NC * 5];
 #define KVS_CK(call) \
     if ((call) != cudaSuccess) return KVS_ERR_CUDA
-    KVS_CP(st, a + A.evict, evict_at_host, (size_t)total_tokens * 4, cudaMemcpyHostToDevice);
-    KVS_CP(st, a + A.cu, cu_seqlens_host, (size_t)(batch + 1) * 4, cudaMemcpyHostToDevice);
-    KVS_CP(st, a + A.q, q_host, A.nq_bytes, cudaMemcpyHostToDevice);
-    KVS_CP(st, a + A.k, k_host, A.nkv_bytes, cudaMemcpyHostToDevice);
-    KVS_CP(st, a + A.v, v_host, A.nkv_bytes, cudaMemcpyHostToDevice);
-    KVS_CK(cudaEventRecord(ev_in, st));                       // dout follows q, k, v on the wire (they are needed first)
-    KVS_CK(cudaStreamWaitEvent(cp, ev_in, 0));
-    KVS_CP(cp, a + A.dout, dout_host, A.nq_bytes, cudaMemcpyHostToDevice);      // overlaps the forward
-    KVS_CK(cudaEventRecord(ev_dout, cp));
+    // rows of `width` bytes, `tokens` of them: host row pitch hp, device row pitch = width
+    auto h2d = [&](cudaStream_t s_, void* dst, const void* src, size_t hoff, size_t hp, size_t width) {
+        return cudaMemcpy2DAsync(dst, width, (const char*)src + hoff, hp, width, (size_t)total_tokens, cudaMemcpyHostToDevice, s_);
+    };
+    auto d2h = [&](cudaStream_t s_, void* dst, size_t hoff, size_t hp, const void* src, size_t width) {
+        return cudaMemcpy2DAsync((char*)dst + hoff, hp, src, width, width, (size_t)total_tokens, cudaMemcpyDeviceToHost, s_);
+    };
+    KVS_CK(cudaMemcpyAsync(a + A.evict, evict_at_host, (size_t)total_tokens * 4, cudaMemcpyHostToDevice, st));
+    KVS_CK(cudaMemcpyAsync(a + A.cu, cu_seqlens_host, (size_t)(batch + 1) * 4, cudaMemcpyHostToDevice, st));
+    KVS_CK(cudaMemsetAsync(a + A.sticky, 0, 4, st));
+    KVS_CK(cudaEventRecord(ev_start, st));                 // the copy streams start after what the caller queued before
+    KVS_CK(cudaStreamWaitEvent(R.in, ev_start, 0));
+    KVS_CK(cudaStreamWaitEvent(R.outs, ev_start, 0));
     int rc = kvs_mask_meta((const int32_t*)(a + A.evict), (const int32_t*)(a + A.cu), batch, total_tokens, max_seqlen, a + A.meta,
                            A.meta_bytes, stream);
     if (rc != KVS_OK) return rc;
-    rc = kvs_attn_fwd(a + A.q, a + A.k, a + A.v, a + A.meta, batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, softmax_scale,
-                      a + A.out, (float*)(a + A.lse), stream);
-    if (rc != KVS_OK) return rc;
-    KVS_CK(cudaEventRecord(ev_fwd, st));
-    KVS_CK(cudaStreamWaitEvent(cp, ev_fwd, 0));
-    KVS_CP(cp, out_host, a + A.out, A.nq_bytes, cudaMemcpyDeviceToHost);         // overlaps the backward
-    KVS_CP(cp, lse_host, a + A.lse, A.lse_bytes, cudaMemcpyDeviceToHost);
-    KVS_CK(cudaEventRecord(ev_out, cp));
-    KVS_CK(cudaStreamWaitEvent(st, ev_dout, 0));
-    rc = kvs_attn_bwd(a + A.dout, a + A.q, a + A.k, a + A.v, a + A.out, (const float*)(a + A.lse), a + A.meta, batch, total_tokens,
-                      max_seqlen, Hq, Hkv, head_dim, softmax_scale, grad_dtype, a + A.dq, a + A.dk, a + A.dv, a + A.ws, A.ws_bytes,
-                      stream);
-    if (rc != KVS_OK) return rc;
-    KVS_CP(st, dq_host, a + A.dq, A.gq_bytes, cudaMemcpyDeviceToHost);
-    KVS_CP(st, dk_host, a + A.dk, A.gkv_bytes, cudaMemcpyDeviceToHost);
-    KVS_CP(st, dv_host, a + A.dv, A.gkv_bytes, cudaMemcpyDeviceToHost);
-    KVS_CK(cudaStreamWaitEvent(st, ev_out, 0));               // the caller's stream ends after every copy
-#undef KVS_CP
+    const size_t hq_pitch = (size_t)Hq * head_dim * 2, hkv_pitch = (size_t)Hkv * head_dim * 2;
+    const size_t wq = (size_t)G * head_dim * 2, wkv = (size_t)head_dim * 2;
+    const size_t gq_pitch = (size_t)Hq * head_dim * gsz, gkv_pitch = (size_t)Hkv * head_dim * gsz;
+    const size_t wgq = (size_t)G * head_dim * gsz, wgkv = (size_t)head_dim * gsz;
+    auto upload = [&](int c) -> int {
+        char* sl = a + A.slot0 + (size_t)(c % A.slots) * A.slot_stride;
+        if (c >= A.slots) KVS_CK(cudaStreamWaitEvent(R.in, ev_down(c - A.slots), 0));     // the slot's previous chunk is finished
+        KVS_CK(h2d(R.in, sl + A.q, q_host, (size_t)c * wq, hq_pitch, wq));
+        KVS_CK(h2d(R.in, sl + A.k, k_host, (size_t)c * wkv, hkv_pitch, wkv));
+        KVS_CK(h2d(R.in, sl + A.v, v_host, (size_t)c * wkv, hkv_pitch, wkv));
+        KVS_CK(cudaEventRecord(ev_qkv(c), R.in));
+        KVS_CK(h2d(R.in, sl + A.dout, dout_host, (size_t)c * wq, hq_pitch, wq));
+        KVS_CK(cudaEventRecord(ev_dout(c), R.in));
+        return KVS_OK;
+    };
+    for (int c = 0; c < A.slots && c < NC; ++c)
+        if ((rc = upload(c)) != KVS_OK) return rc;
+    for (int c = 0; c < NC; ++c) {
+        char* sl = a + A.slot0 + (size_t)(c % A.slots) * A.slot_stride;
+        KVS_CK(cudaStreamWaitEvent(st, ev_qkv(c), 0));
+        rc = kvs_attn_fwd(sl + A.q, sl + A.k, sl + A.v, a + A.meta, batch, total_tokens, max_seqlen, G, 1, head_dim, softmax_scale,
+                          sl + A.out, (float*)(sl + A.lse), stream);
+        if (rc != KVS_OK) return rc;
+        KVS_CK(cudaEventRecord(ev_fwd(c), st));
+        KVS_CK(cudaStreamWaitEvent(R.outs, ev_fwd(c), 0));
+        KVS_CK(d2h(R.outs, out_host, (size_t)c * wq, hq_pitch, sl + A.out, wq));
+        KVS_CK(cudaMemcpyAsync((char*)lse_host + (size_t)c * A.lse_bytes, sl + A.lse, A.lse_bytes, cudaMemcpyDeviceToHost, R.outs));
+        KVS_CK(cudaStreamWaitEvent(st, ev_dout(c), 0));
+        rc = kvs_attn_bwd(sl + A.dout, sl + A.q, sl + A.k, sl + A.v, sl + A.out, (const float*)(sl + A.lse), a + A.meta, batch,
+                          total_tokens, max_seqlen, G, 1, head_dim, softmax_scale, grad_dtype, sl + A.dq, sl + A.dk, sl + A.dv,
+                          sl + A.ws, A.ws_bytes, stream);
+        if (rc != KVS_OK) return rc;
+        fold_status_kernel<<<1, 1, 0, st>>>((const int32_t*)(sl + A.ws), (int32_t*)(a + A.sticky));
+        KVS_CK(cudaEventRecord(ev_bwd(c), st));
+        KVS_CK(cudaStreamWaitEvent(R.outs, ev_bwd(c), 0));
+        KVS_CK(d2h(R.outs, dq_host, (size_t)c * wgq, gq_pitch, sl + A.dq, wgq));
+        KVS_CK(d2h(R.outs, dk_host, (size_t)c * wgkv, gkv_pitch, sl + A.dk, wgkv));
+        KVS_CK(d2h(R.outs, dv_host, (size_t)c * wgkv, gkv_pitch, sl + A.dv, wgkv));
+        KVS_CK(cudaEventRecord(ev_down(c), R.outs));
+        if (c + A.slots < NC && (rc = upload(c + A.slots)) != KVS_OK) return rc;
+    }
+    KVS_CK(cudaStreamWaitEvent(st, ev_down(NC - 1), 0));   // the caller's stream ends after every copy (the out stream is in order)
 #undef KVS_CK
-    int32_t hm[2] = {0, 0}, hw[2] = {0, 0};
+    // status words: the metadata buffer's (mask validation, forward) and the folded workspace status (backward)
+    int32_t hm[2] = {0, 0}, hs = 0;
     if (cudaMemcpyAsync(hm, a + A.meta, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVS_ERR_CUDA;
-    if (cudaMemcpyAsync(hw, a + A.ws, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVS_ERR_CUDA;
+    if (cudaMemcpyAsync(&hs, a + A.sticky, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVS_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return KVS_ERR_CUDA;
     if (hm[1] != KVS_OK) return hm[1];
-    return hw[1];
+    if (hs != KVS_OK) return hs;
+    return KVS_OK;
 }

@@ -294,18 +294,23 @@ def test_argument_errors():
     assert e.value.code == B.KVS_ERR_ALIGNMENT
 
 
-def test_host_buffer_entry_point_matches_device_path():
-    w = W.make_workload(3, shrink=32, Hq=4, Hkv=2, batch=3)
+@pytest.mark.parametrize("Hq,Hkv,grad", [(4, 2, "bf16"), (10, 5, "bf16"), (3, 1, "fp32"), (8, 4, "fp32")])
+def test_host_buffer_entry_point_matches_device_path(Hq, Hkv, grad):
+    # the host path pipelines over KV-head groups (three in flight): more groups than slots, a single group,
+    # both gradient types; every group must come back exactly as the one-shot device path computes it
+    grad = B.GRAD_BF16 if grad == "bf16" else B.GRAD_FP32
+    w = W.make_workload(3, shrink=32, Hq=Hq, Hkv=Hkv, batch=3)
     q, k, v, do = W.make_tensors(w, 9)
     qd, kd, vd, dod = (t.to(DEV) for t in (q, k, v, do))
-    _, out, lse, dq, dk, dv = _run_gpu(w, qd, kd, vd, dod, B.GRAD_BF16)
+    _, out, lse, dq, dk, dv = _run_gpu(w, qd, kd, vd, dod, grad)
     pin = lambda t: t.contiguous().pin_memory()
+    gdt = torch.bfloat16 if grad == B.GRAD_BF16 else torch.float32
     ho, hl = pin(torch.empty_like(q)), pin(torch.empty((w.Hq, w.total_tokens), dtype=torch.float32))
-    hdq, hdk, hdv = pin(torch.empty_like(q)), pin(torch.empty_like(k)), pin(torch.empty_like(v))
-    arena = torch.empty(B.kvs_host_arena_bytes(w.batch, w.total_tokens, w.max_seqlen, w.Hq, w.Hkv, w.d, B.GRAD_BF16),
+    hdq, hdk, hdv = (pin(torch.full(t.shape, float("nan"), dtype=gdt)) for t in (q, k, v))
+    arena = torch.empty(B.kvs_host_arena_bytes(w.batch, w.total_tokens, w.max_seqlen, w.Hq, w.Hkv, w.d, grad),
                         dtype=torch.uint8, device=DEV)
     B.kvs_attn_fwd_bwd_host(pin(torch.from_numpy(w.evict_at)), pin(torch.from_numpy(w.cu_seqlens)), pin(q), pin(k), pin(v), pin(do),
-                            w.max_seqlen, w.softmax_scale, B.GRAD_BF16, ho, hl, hdq, hdk, hdv, arena)
+                            w.max_seqlen, w.softmax_scale, grad, ho, hl, hdq, hdk, hdv, arena)
     assert torch.equal(ho, out.cpu()) and torch.equal(hl, lse.cpu())
     assert torch.equal(hdk, dk.cpu()) and torch.equal(hdv, dv.cpu())
     assert torch.allclose(hdq.float(), dq.cpu().float(), atol=2e-2, rtol=2e-2)

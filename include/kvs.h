@@ -252,7 +252,10 @@ size_t kvs_decode_workspace_bytes(int num_seqs, int Hq, int head_dim, int num_sp
  * One decode step: out[s,h] = softmax_j(scale * q[s,h].k_j) v_j over the live cache of sequence s
  * (query head h reads KV head h / (Hq/Hkv)), lse[s,h] = log sum_j exp(scale * q.k_j).
  * q, out: bf16 [num_seqs, Hq, head_dim]; lse: fp32 [num_seqs, Hq].  Hq/Hkv in {1,2,4,7,8}.
- * A sequence with no live token gets out = 0, lse = -inf.
+ * A sequence with no live token gets out = 0, lse = -inf.  Rows of the cache that no token was
+ * written to (the tail of a sequence's last page) may hold anything, NaN included.
+ * workspace: >= kvs_decode_workspace_bytes(...), 256-byte aligned; its first words are a
+ * {magic, status} header that kvs_device_status() reads (a bounded device wait that expired).
  */
 int kvs_decode_attn(const void* q, const void* k_cache, const void* v_cache,
                     const int32_t* block_table, const int32_t* n_tokens,

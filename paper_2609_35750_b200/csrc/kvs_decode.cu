@@ -8,16 +8,21 @@
 // appending a token takes a page from the free list when the last page is full; decode attention
 // reads exactly the pages the table names.  It never sees a mask.
 //
-// Decode attention is bound by HBM (every live K and V row is read once per step), so the kernel
-// is organised around coalesced 256-byte row reads, not around the tensor cores: one CTA per
-// (split, KV head, sequence); each half-warp reads one K (or V) row per load instruction and
-// serves all G query heads of the group from it; 16-token blocks get one softmax update each;
-// partial results of the warps and of the splits are merged at the end.
+// Decode attention is bound by HBM (every live K and V row is read once per step).  Two kernels
+// produce per-split partial results that a third merges:
+//   decode_partial_kernel  CUDA cores, organised around coalesced 256-byte row reads: one CTA per
+//                          (split, KV head, sequence); each half-warp reads one K (or V) row per load
+//                          instruction and serves all G query heads of the group from it;
+//   decode_tc_kernel       (head_dim 128, G in {4, 7, 8}) the same work with both products on the
+//                          tensor core, because with a wide GQA group the CUDA-core kernel is bound by
+//                          its arithmetic, not by the bytes.
 #include "kvs_common.cuh"
+#include <cstring>
 
 namespace kvs {
 
 constexpr int DEC_THREADS = 128;
+constexpr size_t DEC_WS_HEADER = 256;
 
 struct DecodeParams {
     const __nv_bfloat16* q;          // [S, Hq, D]
@@ -197,6 +202,306 @@ decode_partial_kernel(DecodeParams p) {
             p.part_ml[base * 2 + 0] = M;
             p.part_ml[base * 2 + 1] = L;
         }
+    }
+}
+
+// ---- tensor-core variant (head_dim 128, pages of 8..128 tokens) -----------------------------------
+// With G >= 4 query heads per KV head the CUDA-core kernel above is bound by its arithmetic (every K/V
+// element is multiplied G times in fp32), not by HBM.  Here the two products run on the tensor core in
+// the transposed form, so that the 128 keys of a tile (not the few query heads) fill the 128 rows:
+//   S^T [128 keys x 16] = K [128 x d] (Q_pad [16 x d])^T        A = K tile, B = Q (rows >= G are zero)
+//   O^T [d x 16]      += (V [128 keys x d])^T P^T [128 keys x 16]   A = V tile read MN-major, B = P^T
+// One CTA per (split, KV head, sequence), 4 softmax warps (thread = key in the S^T phase, = output
+// column d in the O^T phase) and one control warp (TMA loads of the tile's pages, MMA issue).  A tile
+// is processed serially; three CTAs per SM overlap one another's loads, MMAs and softmax.  Tensor
+// memory: 32 columns (S^T | O^T).  The per-head maximum over the 128 keys of a tile is a warp
+// reduction plus one exchange through shared memory; the reference maximum moves lazily (threshold
+// 8 in base-2 units), so O^T is rescaled in tensor memory only rarely.
+constexpr int DTC_THREADS = 160;
+#ifndef KVS_DEC_TC_MIN_G
+#define KVS_DEC_TC_MIN_G 4
+#endif
+constexpr int DEC_TC_MIN_G = KVS_DEC_TC_MIN_G;
+struct DtcSmem {
+    static constexpr int OFF_K = 0;                    // [128 keys x 128 d] bf16, two 64-column boxes, 128-byte swizzle
+    static constexpr int OFF_V = 32768;
+    static constexpr int OFF_Q = 65536;                // [16 x 128] bf16, two boxes of [16 x 64]
+    static constexpr int OFF_P = 65536 + 4096;         // P^T as [16 heads x 128 keys] bf16, two boxes of [16 x 64]
+    static constexpr int OFF_BAR = 65536 + 8192;       // 8 mbarriers
+    static constexpr int OFF_MISC = OFF_BAR + 64;      // tmem base, abort flag
+    static constexpr int OFF_WMAX = OFF_MISC + 64;     // [2 buffers][4 warps][16] fp32
+    static constexpr int OFF_WSUM = OFF_WMAX + 512;    // [4 warps][16] fp32
+    static constexpr int TOTAL = OFF_WSUM + 256;
+    static constexpr int DYN_BYTES = TOTAL + 1024;     // slack for the 1024-byte alignment
+};
+
+// order-preserving map float -> int, so that a warp-wide integer max gives the float max
+__device__ __forceinline__ int float_order(float x) {
+    const int i = __float_as_int(x);
+    return i ^ ((i >> 31) & 0x7fffffff);
+}
+__device__ __forceinline__ float float_unorder(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
+
+template <int G, bool PAGED_TMA>
+__global__ void __launch_bounds__(DTC_THREADS, 3)
+decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, DecodeParams p, int32_t* status) {
+    constexpr int D = 128;
+    constexpr int BOX = 16384;                  // one 64-column box of a 128-row tile
+    constexpr uint32_t IDESC_S = make_idesc(16, 0, 0);
+    constexpr uint32_t IDESC_O = make_idesc(16, 1, 0);
+    extern __shared__ uint8_t smem_raw[];
+    const int z = blockIdx.x, g = blockIdx.y, s = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n = p.n_tokens[s];
+    const int ps = p.page_size;
+    const int ppt = 128 / ps;                                   // pages per tile
+    const int ntiles = (n + 127) >> 7;
+    const int per = (ntiles + p.nsplit - 1) / p.nsplit;         // contiguous tiles per split
+    const int t_begin = min(z * per, ntiles), t_end = min(t_begin + per, ntiles);
+    const int my_tiles = t_end - t_begin;
+
+    const uint32_t sraw = smem_u32(smem_raw);
+    const uint32_t sbase = (sraw + 1023u) & ~1023u;
+    uint8_t* sgen = smem_raw + (sbase - sraw);
+    const uint32_t sK = sbase + DtcSmem::OFF_K, sV = sbase + DtcSmem::OFF_V, sQ = sbase + DtcSmem::OFF_Q, sP = sbase + DtcSmem::OFF_P;
+    const uint32_t bars = sbase + DtcSmem::OFF_BAR;
+    const uint32_t bar_full = bars, bar_s = bars + 8, bar_p = bars + 16, bar_free = bars + 24;
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sgen + DtcSmem::OFF_MISC);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + DtcSmem::OFF_MISC + 4);
+    float* s_wmax = reinterpret_cast<float*>(sgen + DtcSmem::OFF_WMAX);
+    float* s_wsum = reinterpret_cast<float*>(sgen + DtcSmem::OFF_WSUM);
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar_full, PAGED_TMA ? 1 : 128);
+        mbar_init(bar_s, 1);
+        mbar_init(bar_p, 128);
+        mbar_init(bar_free, 1);
+        fence_mbar_init();
+    }
+    if (warp == 4) {
+        tmem_alloc(smem_u32(s_tmem), 32);
+        tmem_relinquish();
+    } else {
+        // V starts as zeros (rows no page is loaded into must stay finite: their weight is 0, and 0 x NaN is NaN);
+        // Q: rows 0..G-1 of the 16-row B operand, the rest zero; P^T: rows >= G stay zero for good
+        uint4 zero4 = make_uint4(0, 0, 0, 0);
+        for (int i = tid; i < 32768 / 16; i += 128) reinterpret_cast<uint4*>(sgen + DtcSmem::OFF_V)[i] = zero4;
+        for (int i = tid; i < 8192 / 16; i += 128) reinterpret_cast<uint4*>(sgen + DtcSmem::OFF_Q)[i] = zero4;
+        named_bar_sync(1, 128);
+        // Q row h, 16-byte chunk c (8 elements) of box b: physical chunk c ^ (h % 8) of the 128-byte row
+        for (int i = tid; i < G * 16; i += 128) {
+            const int h = i >> 4, c16 = i & 15, b = c16 >> 3, c = c16 & 7;
+            const uint4 v = *reinterpret_cast<const uint4*>(p.q + ((size_t)s * p.Hq + g * G + h) * D + c16 * 8);
+            *reinterpret_cast<uint4*>(sgen + DtcSmem::OFF_Q + b * 2048 + h * 128 + ((c ^ (h & 7)) << 4)) = v;
+        }
+        fence_proxy_async();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *s_tmem;
+    const uint32_t tmem_S = tmem, tmem_O = tmem + 16;
+
+    if (warp == 4) {
+        // ================= control warp: page loads and MMA issue =================
+        const bool leader = elect_one();
+        const int32_t* bt = p.block_table + (size_t)s * p.max_pages;
+        (void)bt;
+        const uint64_t dK = smem_desc(sK, 16, 1024), dQ = smem_desc(sQ, 16, 1024);
+        const uint64_t dV = smem_desc(sV, BOX, 1024), dP = smem_desc(sP, 16, 1024);
+        for (int it = 0; it < my_tiles; ++it) {
+            const int tt = t_begin + it;
+            const int npages = min(ppt, (n - tt * 128 + ps - 1) / ps);
+            if (PAGED_TMA && it > 0) mbar_wait(bar_free, (it - 1) & 1, abort_flag, status);     // K, V, P^T of the previous tile are consumed
+            if (PAGED_TMA && leader) {
+                mbar_expect_tx(bar_full, (uint32_t)(npages * ps) * 512u);
+                for (int i = 0; i < npages; ++i) {
+                    const int row = bt[tt * ppt + i] * ps;
+                    const uint32_t off = (uint32_t)(i * ps) * 128u;
+                    tma_load_3d(sK + off, &tm_k, 0, g, row, bar_full);
+                    tma_load_3d(sK + BOX + off, &tm_k, 64, g, row, bar_full);
+                    tma_load_3d(sV + off, &tm_v, 0, g, row, bar_full);
+                    tma_load_3d(sV + BOX + off, &tm_v, 64, g, row, bar_full);
+                }
+            }
+            mbar_wait(bar_full, it & 1, abort_flag, status);
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {      // S^T = K Q^T, 16 elements of d per step
+                const uint64_t offk = (uint64_t)(((kk >> 2) * BOX + (kk & 3) * 32) >> 4);
+                const uint64_t offq = (uint64_t)(((kk >> 2) * 2048 + (kk & 3) * 32) >> 4);
+                if (leader) mma_ss(tmem_S, dK + offk, dQ + offq, IDESC_S, kk > 0);
+            }
+            if (leader) mma_commit(bar_s);
+            mbar_wait(bar_p, it & 1, abort_flag, status);
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {           // O^T += V^T P^T, 16 keys per step
+                const uint64_t offp = (uint64_t)(((kk >> 2) * 2048 + (kk & 3) * 32) >> 4);
+                if (leader) mma_ss(tmem_O, dV + (uint64_t)(kk * 128), dP + offp, IDESC_O, (it > 0) || (kk > 0));
+            }
+            if (leader) mma_commit(bar_free);
+        }
+    } else {
+        // ================= softmax warps =================
+        const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+        float m_run[G], l_part[G];
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            m_run[h] = -INFINITY;
+            l_part[h] = 0.f;
+        }
+        // Pages smaller than a swizzle atom (8 rows), e.g. one token per page: the softmax warps fetch the tile
+        // themselves, 16 lanes per 256-byte row (coalesced), with cp.async into the swizzled layout; rows past the
+        // end of the sequence are not fetched and keep their earlier, finite contents (their weight is 0).
+        const int32_t* bt = p.block_table + (size_t)s * p.max_pages;
+        // cache rows of this thread's 16 tokens of a tile (looked up one tile ahead, so that the block-table reads
+        // are not in the way when the tile's buffers become free); -1 = past the end of the sequence
+        long long nrow[16];
+        auto lookup_rows = [&](int tt) {
+            const int nvalid = min(128, n - tt * 128);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int r = warp * 32 + 2 * j + (lane >> 4);
+                const int tok = tt * 128 + r;
+                nrow[j] = (r < nvalid) ? (long long)bt[tok / ps] * ps + tok % ps : -1;
+            }
+        };
+        auto load_tile_rows = [&]() {
+            const int c = lane & 15;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int r = warp * 32 + 2 * j + (lane >> 4);
+                if (nrow[j] >= 0) {
+                    const size_t src = ((size_t)nrow[j] * p.Hkv + g) * D + c * 8;
+                    const uint32_t dst = (uint32_t)((c >> 3) * BOX + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sK + dst), "l"(p.k_cache + src) : "memory");
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sV + dst), "l"(p.v_cache + src) : "memory");
+                }
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            fence_proxy_async();
+            mbar_arrive(bar_full);
+        };
+        if (!PAGED_TMA && my_tiles > 0) {
+            lookup_rows(t_begin);
+            load_tile_rows();
+        }
+        for (int it = 0; it < my_tiles; ++it) {
+            const int tt = t_begin + it;
+            if (!PAGED_TMA && it + 1 < my_tiles) lookup_rows(tt + 1);
+            const int nvalid = min(128, n - tt * 128);
+            const int loaded = min(ppt, (n - tt * 128 + ps - 1) / ps) * ps;
+            mbar_wait(bar_full, it & 1, abort_flag, status);
+            if (PAGED_TMA && tid >= nvalid && tid < loaded) {
+                // rows of the last page past the end of the sequence were never written by anyone
+                const uint4 zero4 = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    *reinterpret_cast<uint4*>(sgen + DtcSmem::OFF_V + tid * 128 + c * 16) = zero4;
+                    *reinterpret_cast<uint4*>(sgen + DtcSmem::OFF_V + BOX + tid * 128 + c * 16) = zero4;
+                }
+            }
+            mbar_wait(bar_s, it & 1, abort_flag, status);
+            tc_fence_after();
+            uint32_t r[16];
+            tmem_ld16(tmem_S + lane_sel, r);
+            tmem_wait_ld();
+            float sc[G];
+            float* wmax = s_wmax + (it & 1) * 64;
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                sc[h] = (tid < nvalid) ? __uint_as_float(r[h]) * p.scale_log2 : -INFINITY;
+                const int wm = __reduce_max_sync(0xffffffffu, float_order(sc[h]));
+                if (lane == 0) wmax[warp * 16 + h] = float_unorder(wm);
+            }
+            named_bar_sync(1, 128);
+            bool grow_any = false;
+            float tmax[G];
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                tmax[h] = fmaxf(fmaxf(wmax[h], wmax[16 + h]), fmaxf(wmax[32 + h], wmax[48 + h]));
+                grow_any |= (tmax[h] > m_run[h] + 8.0f) || (m_run[h] == -INFINITY && tmax[h] > -INFINITY);
+            }
+            if (grow_any) {                      // the same decision in every thread: the maxima are CTA-wide
+                float alpha[16];
+#pragma unroll
+                for (int h = 0; h < 16; ++h) alpha[h] = 1.f;
+#pragma unroll
+                for (int h = 0; h < G; ++h) {
+                    const bool grow = (tmax[h] > m_run[h] + 8.0f) || (m_run[h] == -INFINITY && tmax[h] > -INFINITY);
+                    const float m_new = grow ? tmax[h] : m_run[h];
+                    alpha[h] = (m_new == -INFINITY) ? 1.f : fast_exp2(m_run[h] - m_new);
+                    l_part[h] *= alpha[h];
+                    m_run[h] = m_new;
+                }
+                if (it > 0) {                     // O^T row d = tid: every MMA issued before S^T(it) has completed
+                    uint32_t o[16];
+                    tmem_ld16(tmem_O + lane_sel, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int h = 0; h < 16; ++h) o[h] = __float_as_uint(__uint_as_float(o[h]) * alpha[h]);
+                    tmem_st16(tmem_O + lane_sel, o);
+                    tmem_wait_st();
+                }
+            }
+            // weights of key tid for the G heads -> P^T[h][tid] (bf16), row h of box tid / 64
+            uint8_t* prow = sgen + DtcSmem::OFF_P + (tid >> 6) * 2048 + ((tid & 7) << 1);
+            const int chunk = (tid & 63) >> 3;
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                const float m_use = (m_run[h] == -INFINITY) ? 0.f : m_run[h];
+                const float w = fast_exp2(sc[h] - m_use);
+                l_part[h] += w;
+                *reinterpret_cast<__nv_bfloat16*>(prow + h * 128 + ((chunk ^ (h & 7)) << 4)) = __float2bfloat16(w);
+            }
+            fence_proxy_async();      // P^T (and the zeroed V rows) visible to the tensor core's reads of shared memory
+            tc_fence_before();
+            mbar_arrive(bar_p);
+            if (!PAGED_TMA && it + 1 < my_tiles) {
+                mbar_wait(bar_free, it & 1, abort_flag, status);        // K, V of this tile are consumed
+                load_tile_rows();
+            }
+        }
+        // ---- this split's partial result: O^T (unnormalised), the reference maxima and the sums ----
+        if (my_tiles > 0) {
+            mbar_wait(bar_free, (my_tiles - 1) & 1, abort_flag, status);
+            tc_fence_after();
+        }
+        uint32_t o[16];
+        if (my_tiles > 0) {
+            tmem_ld16(tmem_O + lane_sel, o);
+            tmem_wait_ld();
+        } else {
+#pragma unroll
+            for (int h = 0; h < 16; ++h) o[h] = 0u;
+        }
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            float v = l_part[h];
+#pragma unroll
+            for (int ofs = 16; ofs > 0; ofs >>= 1) v += __shfl_xor_sync(0xffffffffu, v, ofs);
+            if (lane == 0) s_wsum[warp * 16 + h] = v;
+            const size_t base = ((size_t)s * p.Hq + g * G + h) * p.nsplit + z;
+            p.part_o[base * D + tid] = __uint_as_float(o[h]);
+        }
+        named_bar_sync(1, 128);
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            if (tid == h) {
+                const size_t base = ((size_t)s * p.Hq + g * G + h) * p.nsplit + z;
+                p.part_ml[base * 2 + 0] = m_run[h];
+                p.part_ml[base * 2 + 1] = s_wsum[h] + s_wsum[16 + h] + s_wsum[32 + h] + s_wsum[48 + h];
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        __syncwarp();
+        tmem_dealloc(tmem, 32);
     }
 }
 
@@ -421,12 +726,59 @@ extern "C" int kvs_decode_num_splits(int num_seqs, int Hkv, int max_tokens) {
 
 extern "C" size_t kvs_decode_workspace_bytes(int num_seqs, int Hq, int head_dim, int num_splits) {
     if (num_seqs < 0 || Hq <= 0 || head_dim <= 0 || num_splits <= 0) return 0;
-    return align_up(sizeof(float) * (size_t)num_seqs * Hq * num_splits * (head_dim + 2), 256);
+    return DEC_WS_HEADER + align_up(sizeof(float) * (size_t)num_seqs * Hq * num_splits * (head_dim + 2), 256);
+}
+
+// the first 256 bytes of the workspace: {magic, status} as in the backward workspace, so that
+// kvs_device_status() reads it; the partial results follow
+__global__ void decode_header_kernel(int32_t* hdr) {
+    hdr[0] = (int32_t)WS_MAGIC;
+    hdr[1] = KVS_OK;
+}
+
+template <int G, bool PAGED_TMA>
+static int launch_decode_tc(const CUtensorMap& tk, const CUtensorMap& tv, const DecodeParams& p, int32_t* status, cudaStream_t st) {
+    auto kern = decode_tc_kernel<G, PAGED_TMA>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DtcSmem::DYN_BYTES) != cudaSuccess) return KVS_ERR_CUDA;
+    dim3 grid(p.nsplit, p.Hkv, p.S);
+    kern<<<grid, DTC_THREADS, DtcSmem::DYN_BYTES, st>>>(tk, tv, p, status);
+    return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
 }
 
 template <int D>
-static int launch_decode(const DecodeParams& p, int G, void* out, float* lse, cudaStream_t st) {
+static int launch_decode(const DecodeParams& p, int G, const void* k_cache, const void* v_cache, int32_t* status, void* out, float* lse,
+                         cudaStream_t st) {
     dim3 grid(p.nsplit, p.Hkv, p.S);
+    const int ps = p.page_size;
+    // tensor-core variant: head_dim 128 and a GQA group of 4 or more.  Pages that are whole 8-row swizzle atoms and
+    // tile 128 tokens exactly come in by TMA, one box per page; smaller pages (one token per page) by cp.async rows.
+    const bool tc = (D == 128) && (G >= DEC_TC_MIN_G) && (G == 4 || G == 7 || G == 8);
+    const bool paged_tma = (ps % 8 == 0) && (ps <= 128) && (128 % ps == 0);
+    if (tc) {
+        int rc = check_device_sm100();
+        if (rc != KVS_OK) return rc;
+        CUtensorMap tk, tv;
+        memset(&tk, 0, sizeof(tk));
+        memset(&tv, 0, sizeof(tv));
+        if (paged_tma) {
+            // the caches as (d, Hkv, rows) with rows = pages * page_size; the row count is not known here, and the
+            // map only uses it to clip boxes, which never stick out (a box is one page)
+            if ((rc = make_tmap_thd(&tk, k_cache, 1 << 30, p.Hkv, 128, ps)) != KVS_OK) return rc;
+            if ((rc = make_tmap_thd(&tv, v_cache, 1 << 30, p.Hkv, 128, ps)) != KVS_OK) return rc;
+            switch (G) {
+                case 4: rc = launch_decode_tc<4, true>(tk, tv, p, status, st); break;
+                case 7: rc = launch_decode_tc<7, true>(tk, tv, p, status, st); break;
+                default: rc = launch_decode_tc<8, true>(tk, tv, p, status, st); break;
+            }
+        } else {
+            switch (G) {
+                case 4: rc = launch_decode_tc<4, false>(tk, tv, p, status, st); break;
+                case 7: rc = launch_decode_tc<7, false>(tk, tv, p, status, st); break;
+                default: rc = launch_decode_tc<8, false>(tk, tv, p, status, st); break;
+            }
+        }
+        if (rc != KVS_OK) return rc;
+    } else
     switch (G) {
         case 1: decode_partial_kernel<D, 1><<<grid, DEC_THREADS, 0, st>>>(p); break;
         case 2: decode_partial_kernel<D, 2><<<grid, DEC_THREADS, 0, st>>>(p); break;
@@ -467,8 +819,11 @@ extern "C" int kvs_decode_attn(const void* q, const void* k_cache, const void* v
     p.nsplit = num_splits;
     const float s = softmax_scale == 0.f ? 1.0f / sqrtf((float)head_dim) : softmax_scale;
     p.scale_log2 = s * 1.4426950408889634f;
-    p.part_o = (float*)workspace;
+    p.part_o = (float*)((char*)workspace + DEC_WS_HEADER);
     p.part_ml = p.part_o + (size_t)num_seqs * Hq * num_splits * head_dim;
     cudaStream_t st = (cudaStream_t)stream;
-    return head_dim == 64 ? launch_decode<64>(p, Hq / Hkv, out, lse, st) : launch_decode<128>(p, Hq / Hkv, out, lse, st);
+    decode_header_kernel<<<1, 1, 0, st>>>((int32_t*)workspace);
+    int32_t* status = (int32_t*)workspace + 1;
+    return head_dim == 64 ? launch_decode<64>(p, Hq / Hkv, k_cache, v_cache, status, out, lse, st)
+                          : launch_decode<128>(p, Hq / Hkv, k_cache, v_cache, status, out, lse, st);
 }

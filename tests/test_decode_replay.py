@@ -179,3 +179,59 @@ def test_batched_decode_three_sequences_and_error_reporting():
         bad2.append(kk, kk)
     bad2.evict(torch.tensor([(0, 1, 1)], dtype=torch.int32, device="cuda"))        # the half-filled last page
     assert bad2.status()[0] == B.KVS_ERR_INVALID_ARG and int(bad2.n_tokens[0]) == 6
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("G,Hkv,ps", [(4, 2, 16), (8, 1, 16), (7, 2, 8), (8, 2, 32), (4, 1, 128), (8, 1, 64),
+                                      (8, 1, 1), (4, 2, 4), (7, 1, 3), (2, 2, 16), (1, 2, 1)])
+def test_decode_attention_from_a_hand_built_cache(G, Hkv, ps):
+    """Decode attention against its plain definition (softmax over exactly the rows the block table names), on a
+    cache built by hand: scattered pages, lengths that end inside a page / inside a 128-token tile / at zero, and NaN
+    in every row no token was written to (such rows must not leak into the result)."""
+    from paper_2609_35750_b200 import binding as B
+    rng = np.random.default_rng(100 * G + ps)
+    d, Hq = 128, G * Hkv
+    lens = [0, 1, ps - 1, ps, 127, 128, 129, 300, 1000, 1537]
+    S = len(lens)
+    max_pages = (max(lens) + ps - 1) // ps + 1
+    num_pages = sum((n + ps - 1) // ps for n in lens) + 5
+    k_cache = torch.full((num_pages, ps, Hkv, d), float("nan"), dtype=torch.bfloat16)
+    v_cache = torch.full((num_pages, ps, Hkv, d), float("nan"), dtype=torch.bfloat16)
+    table = torch.zeros((S, max_pages), dtype=torch.int32)
+    perm = rng.permutation(num_pages)
+    nxt, rows = 0, []
+    for s, n in enumerate(lens):
+        kk = torch.from_numpy(rng.standard_normal((n, Hkv, d)).astype(np.float32)).to(torch.bfloat16)
+        vv = torch.from_numpy(rng.standard_normal((n, Hkv, d)).astype(np.float32)).to(torch.bfloat16)
+        rows.append((kk, vv))
+        for pi in range((n + ps - 1) // ps):
+            page = int(perm[nxt]); nxt += 1
+            table[s, pi] = page
+            m = min(ps, n - pi * ps)
+            k_cache[page, :m] = kk[pi * ps: pi * ps + m]
+            v_cache[page, :m] = vv[pi * ps: pi * ps + m]
+    q = torch.from_numpy(rng.standard_normal((S, Hq, d)).astype(np.float32)).to(torch.bfloat16)
+    n_tokens = torch.tensor(lens, dtype=torch.int32)
+    cache = B.PagedCache(num_pages, ps, S, max_pages, Hkv, d)
+    cache.k_cache.copy_(k_cache)
+    cache.v_cache.copy_(v_cache)
+    cache.block_table.copy_(table)
+    cache.n_tokens.copy_(n_tokens)
+    for splits in (1, 3):
+        ws = torch.empty(int(B.load().kvs_decode_workspace_bytes(S, Hq, d, splits)), dtype=torch.uint8, device="cuda")
+        out, lse = cache.decode(q.cuda(), num_splits=splits, workspace=ws)
+        assert B.kvs_device_status(ws) == B.KVS_OK
+        out, lse = out.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+        scale = 1.0 / np.sqrt(d)
+        for s, n in enumerate(lens):
+            kk, vv = (t.float().numpy().astype(np.float64) for t in rows[s])
+            for h in range(Hq):
+                if n == 0:
+                    assert np.all(out[s, h] == 0) and lse[s, h] == -np.inf
+                    continue
+                sc = kk[:, h // G] @ q[s, h].float().numpy().astype(np.float64) * scale
+                mx = sc.max()
+                w = np.exp(sc - mx)
+                ref_o, ref_l = (w[:, None] * vv[:, h // G]).sum(0) / w.sum(), mx + np.log(w.sum())
+                assert np.isfinite(out[s, h]).all(), (s, h, n)
+                assert np.abs(out[s, h] - ref_o).max() < 2e-2 and abs(lse[s, h] - ref_l) < 2e-3, (splits, s, h, n)

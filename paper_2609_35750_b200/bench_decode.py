@@ -74,7 +74,7 @@ def main():
                    "Hkv": a.hkv, "head_dim": a.head_dim, "splits": splits,
                    "l2": "K/V working set %.0f MB, larger than L2" % (algo / 1e6)},
         "tokens_per_s": S / (ms * 1e-3),
-        "roofline": {"kernel": ("decode_tc_kernel (tcgen05)" if (a.head_dim == 128 and a.hq // a.hkv in (4, 7, 8)) else "decode_partial_kernel"), "bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
+        "roofline": {"kernel": ("decode_tc_kernel (tcgen05)" if (a.head_dim == 128 and a.hq // a.hkv in (1, 2, 4, 7, 8) and (a.hq // a.hkv >= 4 or (a.page_size % 8 == 0 and 128 % a.page_size == 0))) else "decode_partial_kernel"), "bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
                      "frac": gbs / peak, "traffic": None, "peak_source": src + " copy bandwidth"},
         "dtype": "bf16", "data": "synthetic"}))
 

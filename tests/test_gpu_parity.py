@@ -65,7 +65,7 @@ def _check_meta(w, meta):
     assert np.array_equal(kmax, np.concatenate([b for _, b in mm]))
 
 
-def _full_parity(w, seed=0, tensors=None, bwd=True, dq_abs=None):
+def _full_parity(w, seed=0, tensors=None, bwd=True, dq_abs=None, dkv_abs=None):
     q, k, v, do = tensors if tensors is not None else W.make_tensors(w, seed)
     qd, kd, vd, dod = (t.to(DEV) for t in (q, k, v, do))
     meta, out, lse, dq, dk, dv = _run_gpu(w, qd, kd, vd, dod, B.GRAD_FP32)
@@ -78,15 +78,15 @@ def _full_parity(w, seed=0, tensors=None, bwd=True, dq_abs=None):
         return out, lse, dq, dk, dv
     rdq, rdk, rdv = O.varlen_bwd(qn, kn, vn, don, w.evict_at, w.cu_seqlens, w.scale)
     _close("dq", _f64(dq), rdq, max_abs=dq_abs)
-    _close("dk", _f64(dk), rdk)
-    _close("dv", _f64(dv), rdv)
+    _close("dk", _f64(dk), rdk, max_abs=dkv_abs)
+    _close("dv", _f64(dv), rdv, max_abs=dkv_abs)
     # bf16 gradient outputs: same kernels plus the cast pass
     _, out2, lse2, dq2, dk2, dv2 = _run_gpu(w, qd, kd, vd, dod, B.GRAD_BF16)
     assert dq2.dtype == torch.bfloat16
     assert torch.equal(out, out2) and torch.equal(lse, lse2)       # forward is run-to-run identical
     _close("dq(bf16)", _f64(dq2), rdq, bf16_out=True, max_abs=dq_abs)
-    _close("dk(bf16)", _f64(dk2), rdk, bf16_out=True)
-    _close("dv(bf16)", _f64(dv2), rdv, bf16_out=True)
+    _close("dk(bf16)", _f64(dk2), rdk, bf16_out=True, max_abs=dkv_abs)
+    _close("dv(bf16)", _f64(dv2), rdv, bf16_out=True, max_abs=dkv_abs)
     return out, lse, dq, dk, dv
 
 
@@ -103,13 +103,20 @@ def test_cfg0_full():
     ("cfg4_G8", dict(cfg=4, shrink=32, Hq=8, Hkv=1)),
     ("cfg4b", dict(cfg=4, shrink=32, Hq=8, Hkv=1, variant="b")),
     ("cfg4_control", dict(cfg=4, shrink=32, Hq=8, Hkv=1, variant="control")),
+    ("cfg2_G3", dict(cfg=2, shrink=32, Hq=6, Hkv=2, batch=1)),          # a pair of heads plus a single one per group
+    ("cfg2_G1", dict(cfg=2, shrink=32, Hq=3, Hkv=3, batch=2)),          # no grouping: every forward CTA has one head
+    ("cfg6_G16", dict(cfg=6, shrink=32, Hq=16, Hkv=1, batch=1)),        # non-monotone evict_at, a wide group
 ])
 def test_shrunk_configs_full_tensor(name, kw):
     # Variant B of config 1 folds 1/sqrt(d) into Q and runs with softmax_scale = 1, so dq = 1 * dS k is
     # sqrt(d) times larger than with the default scale (|dq| reaches ~36) and the rounding of dS to bf16
     # alone moves it by more than 2e-2; its absolute bound is scaled by sqrt(d), the relative one is not.
     dq_abs = MAX_ABS * np.sqrt(128.0) if name == "cfg1B_scale1" else None
-    _full_parity(W.make_workload(seed=1, **kw), seed=1, dq_abs=dq_abs)
+    # dk and dv of a KV head sum the bf16-rounded P and dS of its G query heads: with G = 16, twice the widest group
+    # of the configs the 2e-2 bound is stated for, the rounding noise is sqrt(2) times larger (measured 0.0226); the
+    # relative bound stays as it is
+    dkv_abs = MAX_ABS * np.sqrt(2.0) if name == "cfg6_G16" else None
+    _full_parity(W.make_workload(seed=1, **kw), seed=1, dq_abs=dq_abs, dkv_abs=dkv_abs)
 
 
 @pytest.mark.parametrize("seed", [0, 1, 2])

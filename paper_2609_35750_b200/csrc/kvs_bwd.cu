@@ -26,30 +26,58 @@ __host__ __device__ inline BwdWsLayout bwd_ws_layout(int total_tokens, int Hq, i
 }
 
 // ---- pre-pass ---------------------------------------------------------------------------------
+// D[h][tok] = sum_c dout[tok][h][c] * out[tok][h][c], and the fp32 dQ accumulator cleared in the same pass (it is
+// the destination of the main kernel's reduce-adds).  16 bytes per lane and tensor, D/8 lanes per row, DOT_ROWS rows in
+// flight per lane: the pass streams 2 x 2 B in and 4 B out per element and is bound by HBM.
+constexpr int DOT_ROWS = 4;
 template <int D>
-__global__ void bwd_dot_kernel(const __nv_bfloat16* __restrict__ dout, const __nv_bfloat16* __restrict__ out,
-                               float* __restrict__ dvec, int total_tokens, int Hq, WsHeader* hdr) {
+__global__ void __launch_bounds__(256)
+bwd_dot_kernel(const __nv_bfloat16* __restrict__ dout, const __nv_bfloat16* __restrict__ out,
+               float* __restrict__ dvec, float* __restrict__ dq_acc, int total_tokens, int Hq, WsHeader* hdr) {
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         hdr->magic = WS_MAGIC;
         hdr->status = KVS_OK;
     }
-    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    constexpr int LPR = D / 8;                  // lanes per row: 16 or 8
+    constexpr int RPW = 32 / LPR;               // rows per warp and step
+    const long long rows = (long long)total_tokens * Hq;
+    const long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (warp >= (long long)total_tokens * Hq) return;
-    const int tok = (int)(warp / Hq), h = (int)(warp % Hq);
-    constexpr int PER = D / 32;     // 2 or 4 bf16 per lane
-    const __nv_bfloat16* a = dout + (size_t)warp * D + lane * PER;
-    const __nv_bfloat16* b = out + (size_t)warp * D + lane * PER;
-    float acc = 0.f;
+    const int sub = lane / LPR, c = lane % LPR;
+    const long long row0 = gw * (RPW * DOT_ROWS) + sub;
+    uint4 x[DOT_ROWS], y[DOT_ROWS];
 #pragma unroll
-    for (int e = 0; e < PER; e += 2) {
-        const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(a + e));
-        const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(b + e));
-        acc += x.x * y.x + x.y * y.y;
+    for (int r = 0; r < DOT_ROWS; ++r) {
+        const long long row = row0 + (long long)r * RPW;
+        if (row < rows) {
+            x[r] = *reinterpret_cast<const uint4*>(dout + (size_t)row * D + c * 8);
+            y[r] = *reinterpret_cast<const uint4*>(out + (size_t)row * D + c * 8);
+        } else {
+            x[r] = y[r] = make_uint4(0, 0, 0, 0);
+        }
     }
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) dvec[(size_t)h * total_tokens + tok] = acc;
+    for (int r = 0; r < DOT_ROWS; ++r) {
+        const long long row = row0 + (long long)r * RPW;
+        const uint32_t xa[4] = {x[r].x, x[r].y, x[r].z, x[r].w}, ya[4] = {y[r].x, y[r].y, y[r].z, y[r].w};
+        float acc = 0.f;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            acc = fmaf(__uint_as_float(xa[e] << 16), __uint_as_float(ya[e] << 16), acc);
+            acc = fmaf(__uint_as_float(xa[e] & 0xffff0000u), __uint_as_float(ya[e] & 0xffff0000u), acc);
+        }
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (row < rows) {
+            if (dq_acc) {
+                float4* z = reinterpret_cast<float4*>(dq_acc + (size_t)row * D + c * 8);
+                z[0] = zero;
+                z[1] = zero;
+            }
+            if (c == 0) dvec[(size_t)(row % Hq) * total_tokens + (row / Hq)] = acc;
+        }
+    }
 }
 
 // ---- post-pass --------------------------------------------------------------------------------
@@ -529,14 +557,16 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 template <int D>
 static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                       const CUtensorMap& tdq, const MetaView& mv,
-                      const BwdParams& p, const __nv_bfloat16* dout, const __nv_bfloat16* out, float* dvec, WsHeader* hdr,
-                      int nb_cap, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1) {
+                      const BwdParams& p, const __nv_bfloat16* dout, const __nv_bfloat16* out, float* dvec, float* dq_acc,
+                      WsHeader* hdr, int nb_cap, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1) {
     {
-        const long long warps = (long long)p.total_tokens * p.Hq;
+        const long long rows = (long long)p.total_tokens * p.Hq;
+        const int rows_per_warp = (32 / (D / 8)) * DOT_ROWS;
+        const long long warps = (rows + rows_per_warp - 1) / rows_per_warp;
         const int threads = 256;
         const long long blocks = (warps * 32 + threads - 1) / threads;
         if (blocks > 0x7fffffffLL) return KVS_ERR_UNSUPPORTED;
-        bwd_dot_kernel<D><<<(unsigned)blocks, threads, 0, st>>>(dout, out, dvec, p.total_tokens, p.Hq, hdr);
+        bwd_dot_kernel<D><<<(unsigned)(blocks > 0 ? blocks : 1), threads, 0, st>>>(dout, out, dvec, dq_acc, p.total_tokens, p.Hq, hdr);
     }
     auto kern = bwd_kernel<D>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::DYN_BYTES) != cudaSuccess) return KVS_ERR_CUDA;
@@ -600,11 +630,10 @@ extern "C" int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, c
     p.dv = dv;
     p.grad_fp32 = grad_dtype == KVS_GRAD_FP32;
     p.status = &((WsHeader*)ws)->status;
-    if (cudaMemsetAsync(dq_acc, 0, nq * sizeof(float), st) != cudaSuccess) return KVS_ERR_CUDA;
     rc = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, tdq, mv, p, (const __nv_bfloat16*)dout, (const __nv_bfloat16*)out, (float*)(ws + W.dvec),
-                                         (WsHeader*)ws, L.nb_cap, st, ev0, ev1)
+                                         dq_acc, (WsHeader*)ws, L.nb_cap, st, ev0, ev1)
                         : launch_bwd<128>(tq, tk, tv, tdo, tdq, mv, p, (const __nv_bfloat16*)dout, (const __nv_bfloat16*)out,
-                                          (float*)(ws + W.dvec), (WsHeader*)ws, L.nb_cap, st, ev0, ev1);
+                                          (float*)(ws + W.dvec), dq_acc, (WsHeader*)ws, L.nb_cap, st, ev0, ev1);
     if (rc != KVS_OK) return rc;
     if (grad_dtype == KVS_GRAD_BF16) {
         const size_t n4 = nq / 4;

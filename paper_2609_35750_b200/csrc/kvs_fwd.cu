@@ -2,7 +2,9 @@
 //
 // One CTA per (query block, pair of query heads of one GQA group).  The two heads share every K/V
 // tile (identical key-block list and element mask), so each tile is fetched once for two 128-row
-// query tiles.  384 threads in three warp groups:
+// query tiles.  The last head of an odd group (and every head when there is no grouping) gets a CTA
+// of its own, in which the two softmax groups take alternate key blocks of that one head as two
+// independent streams, merged at the end.  384 threads in three warp groups:
 //   warps 0-3   softmax of tile 0 (one query row per thread)        } registers re-balanced with
 //   warps 4-7   softmax of tile 1                                    } setmaxnreg (208 / 208 / 88)
 //   warp 8      producer: TMA for Q0, Q1 and the K and V rings (2 stages each; K runs one key
@@ -78,6 +80,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const int g = blockIdx.y / pairs_per_group;
     const int h0 = g * G + 2 * (blockIdx.y % pairs_per_group);
     const int ntile = (h0 + 1 < (g + 1) * G) ? 2 : 1;       // an odd group ends with a single head
+    // A CTA with a single head still runs both softmax groups: they take alternate key blocks of that head as two
+    // independent streams (own S, O, running maximum and sum), merged at the end like the splits of a split-KV decode.
+    const bool dual = (ntile == 1);
     const int b = mv.blk_trace[gb];
     const int m = gb - mv.blk_off[b];
     const int tok0 = mv.seq_start[b];
@@ -190,14 +195,51 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const uint64_t dK0 = smem_desc(sKV, 16, 1024);
             const uint64_t dV0 = smem_desc(sKV + L::TB, BOX_BYTES, 1024);
             constexpr uint64_t TBU = (uint64_t)(L::TB >> 4);
-            auto issue_s = [&](int t, int s) {
+            auto issue_s_q = [&](int t, int s, int qt) {      // S_t = Q_qt K(stage s)^T
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
-                    if (leader) mma_ss(tmem + t * 128, dQ0 + t * TBU + off, dK0 + s * 2 * TBU + off, IDESC_S, kk > 0);
+                    if (leader) mma_ss(tmem + t * 128, dQ0 + qt * TBU + off, dK0 + s * 2 * TBU + off, IDESC_S, kk > 0);
                 }
                 if (leader) mma_commit(bar_s(t));
             };
+            auto issue_s = [&](int t, int s) { issue_s_q(t, s, t); };
+            if (dual) {
+                // One head, two streams: stream t = key blocks i with i % 2 == t, on S_t / O_t and ring stage t.
+                if (nlist > 0) {
+                    mbar_wait(bar_q, 0, abort_flag, status);
+                    for (int t = 0; t < 2 && t < nlist; ++t) {
+                        mbar_wait(bar_kfull(t), 0, abort_flag, status);
+                        tc_fence_after();
+                        issue_s_q(t, t, 0);
+                        if (leader) mma_commit(bar_kfree(t));
+                    }
+                }
+                for (int i = 0; i < nlist; ++i) {
+                    const int t = i & 1;
+                    const uint32_t ph = (uint32_t)(i >> 1) & 1;
+                    mbar_wait(bar_p0(t), ph, abort_flag, status);
+                    mbar_wait(bar_vfull(t), ph, abort_flag, status);
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < P_SPLIT / 16; ++kk)
+                        if (leader) mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, dV0 + t * 2 * TBU + (uint64_t)(kk * 128), IDESC_O,
+                               (i > 1) || (kk > 0));
+                    mbar_wait(bar_p(t), ph, abort_flag, status);
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = P_SPLIT / 16; kk < TILE / 16; ++kk)
+                        if (leader) mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, dV0 + t * 2 * TBU + (uint64_t)(kk * 128), IDESC_O, true);
+                    if (leader) mma_commit(bar_vfree(t));
+                    if (i + 2 < nlist) {
+                        mbar_wait(bar_kfull(t), (uint32_t)((i + 2) >> 1) & 1, abort_flag, status);
+                        tc_fence_after();
+                        issue_s_q(t, t, 0);
+                        if (leader) mma_commit(bar_kfree(t));
+                    }
+                }
+                if (leader) mma_commit(bar_done);
+            } else {
             if (nlist > 0) {
                 mbar_wait(bar_q, 0, abort_flag, status);
                 mbar_wait(bar_kfull(0), 0, abort_flag, status);
@@ -243,28 +285,30 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 }
             }
             if (leader) mma_commit(bar_done);
+            }
         }
     } else {
         // ================= softmax groups =================
         reg_inc<208>();
-        const int t = warp >> 2;                                  // which query tile / head
-        if (t < ntile) {
+        const int t = warp >> 2;                                  // which query tile / head (or stream of the single head)
+        if (t < ntile || dual) {
             const int quad = warp & 3;
             const int row = quad * 32 + lane;                     // query row of the tile == TMEM lane
             const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
             const uint32_t tmem_S = tmem + t * 128 + lane_sel;
             const uint32_t tmem_O = tmem + 256 + t * 128 + lane_sel;
-            const int h = h0 + t;
+            const int h = dual ? h0 : h0 + t;
             const int qi = m * TILE + row;                        // trace-local query index
             float ref_max = -INFINITY;                            // base-2 domain; the exponent's reference
             float run_sum = 0.f;
 
-            for (int i = 0; i < nlist; ++i) {
+            for (int i = dual ? t : 0; i < nlist; i += dual ? 2 : 1) {
                 const int s = i & 1;
                 const int n = list[i];
+                const int it = dual ? (i >> 1) : i;               // how many key blocks this group has done before
                 mbar_wait(bar_evfull(s), (i >> 1) & 1, abort_flag, status);
                 const bool need_mask = sFlag[s] != 0;
-                mbar_wait(bar_s(t), i & 1, abort_flag, status);
+                mbar_wait(bar_s(t), it & 1, abort_flag, status);
                 tc_fence_after();
                 if (tid == 0) KVS_TRF(i, 8);
                 if (tid == 128) KVS_TRF(i, 13);
@@ -318,7 +362,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     const float alpha = (new_ref == -INFINITY) ? 1.f : fast_exp2(ref_max - new_ref);   // ref_max = -inf -> 0
                     run_sum *= alpha;
                     ref_max = new_ref;
-                    if (i > 0) {
+                    if (it > 0) {
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c) {
                             uint32_t r[32];
@@ -383,6 +427,38 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             mbar_wait(bar_done, 0, abort_flag, status);
             tc_fence_after();
             const bool valid = qi < T;
+            // single head: stream 1 hands its partial result (O1 column by column, reference, sum) to stream 0
+            // through the K/V ring's shared memory, which nothing uses any more
+            float* x_o = reinterpret_cast<float*>(sgen + L::OFF_KV);           // [D][128 rows]
+            float* x_ms = x_o + D * TILE;                                     // [2][128 rows]
+            const bool has1 = dual && nlist > 1;
+            float a0 = 1.f, a1 = 0.f;
+            if (dual) {
+                if (t == 1) {
+                    if (has1) {
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t r[32];
+                            tmem_ld32(tmem_O + c * 32, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) x_o[(c * 32 + e) * TILE + row] = __uint_as_float(r[e]);
+                        }
+                    }
+                    x_ms[row] = ref_max;
+                    x_ms[TILE + row] = run_sum;
+                }
+                named_bar_sync(2, 256);
+                if (t == 0) {
+                    const float ref1 = has1 ? x_ms[row] : -INFINITY, sum1 = has1 ? x_ms[TILE + row] : 0.f;
+                    const float mm = fmaxf(ref_max, ref1);
+                    a0 = (ref_max == -INFINITY) ? 0.f : fast_exp2(ref_max - mm);
+                    a1 = (ref1 == -INFINITY) ? 0.f : fast_exp2(ref1 - mm);
+                    run_sum = run_sum * a0 + sum1 * a1;
+                    ref_max = mm;
+                }
+            }
+            if (!dual || t == 0) {
             const float inv = (run_sum > 0.f && nlist > 0) ? 1.f / run_sum : 0.f;
             __nv_bfloat16* orow = p.out + ((size_t)(tok0 + qi) * p.Hq + h) * D;
 #pragma unroll
@@ -393,6 +469,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 if (nlist == 0) {      // only a bad evict_at (already reported by the metadata pass) gets here
 #pragma unroll
                     for (int e = 0; e < 32; ++e) r[e] = 0u;
+                }
+                if (dual) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        float o = __uint_as_float(r[e]) * a0;
+                        if (a1 > 0.f) o = fmaf(x_o[(c * 32 + e) * TILE + row], a1, o);
+                        r[e] = __float_as_uint(o);
+                    }
                 }
                 if (valid) {
                     uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
@@ -408,6 +492,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 }
             }
             if (valid) p.lse[(size_t)h * p.total_tokens + tok0 + qi] = ref_max * 0.6931471805599453f + logf(run_sum);
+            }
         }
     }
     // a Q load whose CTA had no key block to walk is drained before the CTA leaves

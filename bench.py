@@ -7,7 +7,17 @@ One step = kvs_mask_meta + kvs_attn_fwd + kvs_attn_bwd (bf16 gradients, i.e. inc
 row-sum pre-pass and the cast post-pass) over one synthetic batch resident in HBM.  Prints
 ONE JSON line.  `value` = effective TFLOP/s counting only unmasked (query, key) pairs:
 14 * head_dim * Hq * pairs per step.  With N > 1 every rank runs its own batch of the same
-configuration (seed + rank): independent traces, no collective on the data path.
+configuration (seed + rank): independent traces, no collective on the data path; started
+without a launcher (`python bench.py --gpus N`, WORLD_SIZE unset) it starts the N ranks itself.
+
+After the headline measurement of the default run (config 2, one GPU) the other configurations
+are timed for a few steps each and reported under `per_config` in the same line.
+
+Smaller runs for profilers and other paths, all through the same library calls:
+    --shrink S [--hq H --hkv H --batch B]   a shrunk copy of the configuration
+    --path meta                             the mask-metadata pass alone (large batches: its bandwidth)
+    --path decode [--seqs --live --page-size --hq --hkv --head-dim --splits]
+                                            rollout side: decode attention over a fragmented paged cache
 """
 from __future__ import annotations
 
@@ -27,10 +37,18 @@ if ROOT not in sys.path:
 
 METRIC = "masked_attn_fwd_bwd_effective_tflops"
 UNIT = "TFLOP/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the backward main kernel, from the
-# ncu captures summarised under profiles/ (None until a capture of that workload exists)
-NCU_DRAM_BYTES_PER_LAUNCH = {"cfg2_keep_last_4_turns": 20461770496}   # profiles/bwd_kernel_cfg2.md, full-size light pass
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the backward main kernel: a small JSON
+# file written beside the ncu summaries whenever that kernel is captured (absent or no entry: null)
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "bwd_kernel_traffic.json")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_traffic(workload_name):
+    try:
+        with open(TRAFFIC_FILE) as f:
+            return int(json.load(f)[workload_name]["dram_bytes_per_launch"])
+    except Exception:
+        return None
 
 
 def load_peaks():
@@ -202,63 +220,22 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=2, help="workload 0..4 (default 2: keep-last-4-turns, the target config)")
-    ap.add_argument("--variant", type=str, default="")
-    ap.add_argument("--impl", type=str, default="native", choices=["native", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--cpu-seconds", type=float, default=12.0)
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 0)
-
-    if args.impl == "reference":
-        run_reference(args)
-        return
-
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-
-    # CPU baseline first (rank 0, N = 1 only), before this process touches CUDA
-    cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu_baseline = time_oracle(args.config, args.variant, 0, args.cpu_seconds)
-        cpu_baseline = {k: cpu_baseline[k] for k in ("value", "unit", "cores", "kind", "sample")}
-
-    import torch
-    from paper_2609_35750_b200 import binding as B
-    from paper_2609_35750_b200 import dist as D
-    from paper_2609_35750_b200 import workloads as W
-
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU implementation")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    D.init_from_env(backend="nccl")
-    B.load()
-
-    w = W.make_workload(args.config, seed=rank, variant=args.variant)
-    q, k, v, do = W.make_tensors(w, seed=rank, device=str(dev))
+def time_train_steps(torch, B, W, w, seed, dev, steps, warmup, grad, barrier=None, sampler=None):
+    """Mask metadata + forward + backward, `warmup` untimed and `steps` timed steps on the current stream.
+    Returns a dict of per-phase mean times (ms), the total, and the device status."""
+    q, k, v, do = W.make_tensors(w, seed=seed, device=str(dev))
     ev = torch.from_numpy(w.evict_at).to(dev)
     cu = torch.from_numpy(w.cu_seqlens).to(dev)
     Tt, Hq, Hkv, d = w.total_tokens, w.Hq, w.Hkv, w.d
-    grad = B.GRAD_BF16
     meta = torch.empty(B.kvs_mask_meta_bytes(w.batch, Tt, w.max_seqlen), dtype=torch.uint8, device=dev)
     ws = torch.empty(B.kvs_attn_bwd_workspace_bytes(Tt, Hq, Hkv, d, grad), dtype=torch.uint8, device=dev)
+    gdt = torch.bfloat16 if grad == B.GRAD_BF16 else torch.float32
     out = torch.empty_like(q)
     lse = torch.empty((Hq, Tt), dtype=torch.float32, device=dev)
-    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    dq, dk, dv = (torch.empty(t.shape, dtype=gdt, device=dev) for t in (q, k, v))
     stream = torch.cuda.current_stream()
-
-    n_ev = args.steps
-    ev_fwd = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
-    ev_bwd = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
-    ev_meta = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
+    mk = lambda: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    ev_fwd, ev_bwd, ev_meta = mk(), mk(), mk()
     for pair in ev_bwd:              # create the handles before they are passed through the C ABI
         pair[0].record(stream)
         pair[1].record(stream)
@@ -276,52 +253,254 @@ def main():
         B.kvs_attn_bwd(do, q, k, v, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale, grad, dq=dq, dk=dk, dv=dv,
                        workspace=ws, main_events=(ev_bwd[i] if i is not None else None))
 
-    for _ in range(max(args.warmup, 0)):
+    for _ in range(max(warmup, 0)):
         step()
     torch.cuda.synchronize()
     status = (B.kvs_device_status(meta), B.kvs_device_status(ws))
     if status != (0, 0):
         raise SystemExit(f"device status after warm-up: {status}")
-
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
+    if sampler is not None:
         sampler.start()
         time.sleep(0.3)
-    D.barrier()
+    if barrier is not None:
+        barrier()
     torch.cuda.synchronize()
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_begin.record(stream)
-    for i in range(args.steps):
+    for i in range(steps):
         step(i)
     t_end.record(stream)
     torch.cuda.synchronize()
-    D.barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    ms_total = t_begin.elapsed_time(t_end)
-    ms_total_max, units_total = D.aggregate(ms_total, float(W.fwd_bwd_flops(w)) * args.steps, device=dev)
-    _, tokens_total = D.aggregate(ms_total, float(Tt) * args.steps, device=dev)
+    if barrier is not None:
+        barrier()
+    clocks = sampler.stop() if sampler is not None else None
     status = (B.kvs_device_status(meta), B.kvs_device_status(ws))
     if status != (0, 0):
         raise SystemExit(f"device status after the timed region: {status}")
+    mean = lambda evs: float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    return {"ms_total": t_begin.elapsed_time(t_end), "ms_fwd": mean(ev_fwd), "ms_bwd_main": mean(ev_bwd), "ms_meta": mean(ev_meta),
+            "clocks": clocks, "tensors": (q, k, v, do)}
 
-    ms_fwd = float(np.mean([a.elapsed_time(b) for a, b in ev_fwd]))
-    ms_bwd_main = float(np.mean([a.elapsed_time(b) for a, b in ev_bwd]))
-    ms_meta = float(np.mean([a.elapsed_time(b) for a, b in ev_meta]))
+
+def run_per_config(torch, B, W, dev, peaks, gpu_index):
+    """The other configurations on the same clock as the headline: 1 warm-up + 3 timed steps each."""
+    res = {}
+    for key, cfg, variant in (("0", 0, ""), ("1", 1, ""), ("3", 3, ""), ("4", 4, ""), ("4_control", 4, "control")):
+        w = W.make_workload(cfg, seed=0, variant=variant)
+        sampler = ClockSampler(gpu_index)
+        r = time_train_steps(torch, B, W, w, 0, dev, steps=3, warmup=1, grad=B.GRAD_BF16, sampler=sampler)
+        r.pop("tensors")
+        torch.cuda.empty_cache()
+        ms = r["ms_total"] / 3
+        tf = W.fwd_bwd_flops(w) / (ms * 1e-3) / 1e12
+        res[key] = {"workload": w.name, "tokens": w.total_tokens, "unmasked_pairs": W.count_pairs(w), "steps": 3, "warmup": 1,
+                    "ms_per_step": ms, "effective_tflops": tf, "frac_of_burst_peak": tf / float(peaks["bf16_tflops"]),
+                    "tokens_per_s": w.total_tokens / (ms * 1e-3), "ms_fwd": r["ms_fwd"], "ms_bwd_main": r["ms_bwd_main"],
+                    "sm_mhz_median": (r["clocks"] or {}).get("sm_mhz"), "reasons": (r["clocks"] or {}).get("reasons")}
+    return res
+
+
+def run_meta_only(args):
+    """--path meta: the mask-metadata pass alone (no q/k/v), so that the batch can be large enough for its bandwidth to show."""
+    import torch
+    from paper_2609_35750_b200 import binding as B
+    from paper_2609_35750_b200 import workloads as W
+    dev = "cuda"
+    w = W.make_workload(args.config, seed=0, shrink=args.shrink, Hq=args.hq, Hkv=args.hkv, variant=args.variant, batch=args.batch)
+    ev = torch.from_numpy(w.evict_at).to(dev)
+    cu = torch.from_numpy(w.cu_seqlens).to(dev)
+    nbytes = B.kvs_mask_meta_bytes(w.batch, w.total_tokens, w.max_seqlen)
+    meta = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    ms = []
+    for _ in range(args.warmup + max(args.steps, 1)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.kvs_mask_meta(ev, cu, w.max_seqlen, meta_buf=meta)
+        e1.record()
+        torch.cuda.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    ms = ms[args.warmup:]
+    st = B.kvs_device_status(meta)
+    lens = (w.cu_seqlens[1:] - w.cu_seqlens[:-1]).astype(np.int64)
+    nb = int(((lens + 127) // 128).sum())
+    tiles = int((((lens + 127) // 128) ** 2).sum())
+    # algorithmic bytes: evict_at read once and copied once (4 + 4 B per token), one class byte and one
+    # 2-byte list slot per tile of the per-trace square
+    alg = 8 * w.total_tokens + 3 * tiles
+    peaks = load_peaks()
+    gbs = alg / (float(np.median(ms)) * 1e-3) / 1e9
+    print(json.dumps({"metric": "mask_meta_gbs", "value": gbs, "unit": "GB/s", "steps": len(ms), "warmup": args.warmup,
+                      "ms_per_step": float(np.median(ms)), "config": {"workload": w.name, "traces": w.batch, "tokens": w.total_tokens,
+                                                                       "key_blocks": nb, "tiles": tiles, "meta_buffer_bytes": nbytes},
+                      "roofline": {"kernel": "mask metadata (4 launches)", "bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]),
+                                   "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]), "traffic": None,
+                                   "algorithmic_bytes": alg},
+                      "status": st, "dtype": "int32", "data": "synthetic"}), flush=True)
+    if st != 0:
+        raise SystemExit(1)
+
+
+def run_decode(args):
+    """--path decode: one step = kvs_decode_attn for one new token of every sequence over its live cache.  The kernel
+    reads every live K and V row once, so it is bound by HBM: algorithmic bytes = live K and V rows of the sequences'
+    KV heads.  The block tables point at randomly permuted pages, the state of a cache after many evictions."""
+    import torch
+    from paper_2609_35750_b200 import binding as B
+    dev = "cuda"
+    hq, hkv = args.hq or 28, args.hkv or 4
+    S, n, ps = args.seqs, args.live, args.page_size
+    pages_per_seq = (n + ps - 1) // ps
+    num_pages = S * pages_per_seq + 8
+    cache = B.PagedCache(num_pages, ps, S, pages_per_seq, hkv, args.head_dim, device=dev)
+    g = torch.Generator(device=dev).manual_seed(0)
+    cache.k_cache.copy_(torch.randn(cache.k_cache.shape, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16))
+    cache.v_cache.copy_(torch.randn(cache.v_cache.shape, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16))
+    perm = torch.randperm(num_pages, generator=g, device=dev)[: S * pages_per_seq].to(torch.int32)
+    cache.block_table.copy_(perm.view(S, pages_per_seq))
+    cache.n_tokens.fill_(n)
+    q = torch.randn((S, hq, args.head_dim), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    splits = args.splits or int(B.load().kvs_decode_num_splits(S, hkv, n))
+    ws = torch.empty(int(B.load().kvs_decode_workspace_bytes(S, hq, args.head_dim, splits)), dtype=torch.uint8, device=dev)
+    out = torch.empty_like(q)
+    lse = torch.empty((S, hq), dtype=torch.float32, device=dev)
+    for _ in range(max(args.warmup, 1)):
+        cache.decode(q, num_splits=splits, out=out, lse=lse, workspace=ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        cache.decode(q, num_splits=splits, out=out, lse=lse, workspace=ws)
+    e1.record()
+    torch.cuda.synchronize()
+    if B.kvs_device_status(ws) != 0:
+        raise SystemExit("device status after the timed region: %d" % B.kvs_device_status(ws))
+    ms = e0.elapsed_time(e1) / args.steps
+    algo = 2.0 * S * n * hkv * args.head_dim * 2          # K and V rows, bf16
+    peaks = load_peaks()
+    gbs = algo / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "decode_attn_hbm_gbs", "value": gbs, "unit": "GB/s", "ms_per_step": ms, "steps": args.steps, "warmup": args.warmup,
+        "config": {"workload": "decode over a fragmented paged cache", "seqs": S, "live_tokens": n, "page_size": ps, "Hq": hq,
+                   "Hkv": hkv, "head_dim": args.head_dim, "splits": splits,
+                   "l2": "K/V working set %.0f MB, larger than L2" % (algo / 1e6)},
+        "tokens_per_s": S / (ms * 1e-3),
+        "roofline": {"kernel": "decode attention (partial + combine)", "bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]),
+                     "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]), "traffic": None,
+                     "peak_source": peaks["_source"] + " copy bandwidth"},
+        "dtype": "bf16", "data": "synthetic"}), flush=True)
+
+
+def spawn_ranks(n):
+    """`python bench.py --gpus N` without a launcher: start the N ranks here (one process per GPU, LOCAL_RANK = GPU
+    index), pass rank 0's JSON line through, everything else the ranks print goes to stderr."""
+    from paper_2609_35750_b200 import dist as D
+    results = D.spawn_local(n, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:],
+                            env_extra={"NCCL_DEBUG": os.environ.get("NCCL_DEBUG", "INFO"),
+                                       "NCCL_DEBUG_SUBSYS": os.environ.get("NCCL_DEBUG_SUBSYS", "INIT")})
+    line = None
+    for rank, (rc, text) in enumerate(results):
+        for ln in text.splitlines():
+            if rank == 0 and ln.startswith("{") and '"metric"' in ln:
+                line = ln
+            else:
+                print(f"[rank {rank}] {ln}", file=sys.stderr)
+    bad = [(r, rc) for r, (rc, _) in enumerate(results) if rc != 0]
+    if bad:
+        raise SystemExit(f"bench.py --gpus {n}: ranks failed (rank, exit code): {bad}")
+    if line is None:
+        raise SystemExit(f"bench.py --gpus {n}: rank 0 printed no result line")
+    print(line, flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=2, help="workload 0..7 (default 2: keep-last-4-turns, the target config)")
+    ap.add_argument("--variant", type=str, default="")
+    ap.add_argument("--impl", type=str, default="native", choices=["native", "reference"])
+    ap.add_argument("--path", type=str, default="train", choices=["train", "meta", "decode"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--shrink", type=int, default=1, help="divide every length of the configuration (small cases for profilers)")
+    ap.add_argument("--hq", type=int, default=None)
+    ap.add_argument("--hkv", type=int, default=None)
+    ap.add_argument("--batch", type=int, default=None, help="number of traces (default: the configuration's own)")
+    ap.add_argument("--grad", type=str, default="bf16", choices=["bf16", "fp32"])
+    ap.add_argument("--seqs", type=int, default=64, help="--path decode: sequences")
+    ap.add_argument("--live", type=int, default=7168, help="--path decode: live tokens per sequence")
+    ap.add_argument("--page-size", type=int, default=16, help="--path decode: tokens per page")
+    ap.add_argument("--head-dim", type=int, default=128, help="--path decode")
+    ap.add_argument("--splits", type=int, default=0, help="--path decode: KV splits (0: chosen by the library)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    if args.path == "meta":
+        run_meta_only(args)
+        return
+    if args.path == "decode":
+        run_decode(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args.gpus)
+        return
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    small = args.shrink != 1 or args.hq is not None or args.hkv is not None or args.batch is not None
+
+    # CPU baseline first (rank 0, N = 1 only), before this process touches CUDA
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not small:
+        cpu_baseline = time_oracle(args.config, args.variant, 0, args.cpu_seconds)
+        cpu_baseline = {k: cpu_baseline[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    import torch
+    from paper_2609_35750_b200 import binding as B
+    from paper_2609_35750_b200 import dist as D
+    from paper_2609_35750_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    D.init_from_env(backend="nccl")
+    B.load()
+
+    w = W.make_workload(args.config, seed=rank, variant=args.variant, shrink=args.shrink, Hq=args.hq, Hkv=args.hkv, batch=args.batch)
+    Tt, Hq, Hkv, d = w.total_tokens, w.Hq, w.Hkv, w.d
+    grad = B.GRAD_BF16 if args.grad == "bf16" else B.GRAD_FP32
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    r = time_train_steps(torch, B, W, w, rank, dev, args.steps, args.warmup, grad, barrier=D.barrier, sampler=sampler)
+    q, k, v, do = r.pop("tensors")
+    clocks = r["clocks"]
+    ms_total = r["ms_total"]
+    ms_total_max, units_total = D.aggregate(ms_total, float(W.fwd_bwd_flops(w)) * args.steps, device=dev)
+    _, tokens_total = D.aggregate(ms_total, float(Tt) * args.steps, device=dev)
+    ms_fwd, ms_bwd_main, ms_meta = r["ms_fwd"], r["ms_bwd_main"], r["ms_meta"]
     pairs = W.count_pairs(w)
+    torch.cuda.empty_cache()
 
     # ---- end to end through the C ABI with host buffers ------------------------------------------
     e2e = None
-    if not args.no_e2e:
-        del out, lse, dq, dk, dv, ws, meta
-        torch.cuda.empty_cache()
+    if not args.no_e2e and not small:
         pin = lambda t: t.cpu().contiguous().pin_memory()
         hq, hk, hv, hdo = pin(q), pin(k), pin(v), pin(do)
         hev, hcu = pin(torch.from_numpy(w.evict_at)), pin(torch.from_numpy(w.cu_seqlens))
+        gdt = torch.bfloat16 if grad == B.GRAD_BF16 else torch.float32
         ho = torch.empty(hq.shape, dtype=torch.bfloat16).pin_memory()
         hl = torch.empty((Hq, Tt), dtype=torch.float32).pin_memory()
-        hdq = torch.empty(hq.shape, dtype=torch.bfloat16).pin_memory()
-        hdk = torch.empty(hk.shape, dtype=torch.bfloat16).pin_memory()
-        hdv = torch.empty(hk.shape, dtype=torch.bfloat16).pin_memory()
+        hdq = torch.empty(hq.shape, dtype=gdt).pin_memory()
+        hdk = torch.empty(hk.shape, dtype=gdt).pin_memory()
+        hdv = torch.empty(hk.shape, dtype=gdt).pin_memory()
         del q, k, v, do
         torch.cuda.empty_cache()
         arena = torch.empty(B.kvs_host_arena_bytes(w.batch, Tt, w.max_seqlen, Hq, Hkv, d, grad), dtype=torch.uint8, device=dev)
@@ -346,23 +525,31 @@ def main():
         e2e = {"value": units_e2e / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e / e_steps, "steps": e_steps,
                "api": "kvs_attn_fwd_bwd_host (pinned host buffers in, pinned host buffers out)"}
+        del arena, hq, hk, hv, hdo, ho, hl, hdq, hdk, hdv
+        torch.cuda.empty_cache()
+    else:
+        del q, k, v, do
+        torch.cuda.empty_cache()
 
     if rank != 0:
         D.shutdown()
         return
 
     peaks = load_peaks()
+    per_config = None
+    if world == 1 and not small and args.config == 2 and args.variant == "" and not args.no_per_config:
+        per_config = run_per_config(torch, B, W, dev, peaks, local_rank)
+
     value = units_total / (ms_total_max * 1e-3) / 1e12
     flops_bwd_main = 10.0 * d * Hq * pairs
     achieved = flops_bwd_main / (ms_bwd_main * 1e-3) / 1e12
     peak = float(peaks["bf16_tflops_sustained"])      # the kernel is timed inside a long step
-    profile_traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(w.name)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_total_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "traces": w.batch, "tokens": Tt, "Hq": Hq, "Hkv": Hkv, "head_dim": d,
-                   "unmasked_pairs": pairs, "flops_per_step": W.fwd_bwd_flops(w), "grad_dtype": "bf16",
+                   "unmasked_pairs": pairs, "flops_per_step": W.fwd_bwd_flops(w), "grad_dtype": args.grad,
                    "l2": "inputs larger than L2 (q, dout, out, dq are each %.2f GB)" % (Tt * Hq * d * 2 / 1e9),
                    "parallelism": f"independent batches x{world}" if world > 1 else "single GPU", "notes": w.notes},
         "tokens_per_s": tokens_total / (ms_total_max * 1e-3),
@@ -373,13 +560,15 @@ def main():
                          "bwd_pre_post": ms_total_max / args.steps - ms_meta - ms_fwd - ms_bwd_main,
                          "fwd_tflops": 4.0 * d * Hq * pairs / (ms_fwd * 1e-3) / 1e12, "bwd_main_tflops": achieved},
         "roofline": {"kernel": "bwd_kernel (dQ/dK/dV main)", "bound": "tensor", "achieved": achieved, "peak": peak,
-                     "unit": "TFLOP/s", "frac": achieved / peak, "traffic": profile_traffic,
+                     "unit": "TFLOP/s", "frac": achieved / peak, "traffic": load_traffic(w.name),
+                     "frac_of_burst_peak": achieved / float(peaks["bf16_tflops"]),
                      "peak_source": f"{peaks['_source']} cuBLAS bf16, sustained (kernel timed inside a long step)",
                      "flops_per_launch": flops_bwd_main},
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": 8 * args.steps,
+        "gpu_launches": (8 if grad == B.GRAD_BF16 else 7) * args.steps,
         "cpu_baseline": cpu_baseline,
+        "per_config": per_config,
     }
     print(json.dumps(line), flush=True)
     D.shutdown()

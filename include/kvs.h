@@ -104,7 +104,9 @@ int kvs_mask_meta_export(const void* meta_buf, int batch, const int32_t* cu_seql
                          kvs_stream_t stream);
 
 /*
- * Forward:  S_ij = scale * q_i.k_j over allowed j;  lse_i = log sum_j exp S_ij;
+ * Forward of the trainer-side attention (Sec. 2, "KV-streams" paragraph; Fig. 2 caption: one continuous
+ * trace, the mask hides the deleted span, one forward pass reproduces the rollout's evictions):
+ *           S_ij = scale * q_i.k_j over allowed j;  lse_i = log sum_j exp S_ij;
  *           out_i = sum_j exp(S_ij - lse_i) v_j.   Query head h reads KV head h / (Hq/Hkv).
  * EMPTY tiles are never loaded; element masks are evaluated on PARTIAL tiles only.
  * softmax_scale == 0 selects 1/sqrt(head_dim).  bf16 operands, fp32 accumulation.
@@ -114,11 +116,28 @@ int kvs_attn_fwd(const void* q, const void* k, const void* v, const void* meta_b
                  int Hq, int Hkv, int head_dim, float softmax_scale,
                  void* out, float* lse, kvs_stream_t stream);
 
+/*
+ * Student and teacher forward in one pass (App. D.3 "Training Objectives", self-distillation: the
+ * student is conditioned under the eviction mask, the teacher is a full-context pass of the same
+ * model on the same tokens).  Both use the same q, k, v:
+ *     student:  kvs_attn_fwd's result (query i reads key j iff j <= i < evict_at[j])
+ *     teacher:  plain causal attention over the same trace (query i reads every key j <= i)
+ * Every S = q k^T tile is formed once and feeds both softmax / P V streams; a key block that is EMPTY
+ * for the student costs the student nothing.  Arguments as kvs_attn_fwd, with one (out, lse) pair per
+ * stream; all four are overwritten.  meta_buf is the one kvs_mask_meta built for the eviction mask.
+ */
+int kvs_attn_fwd_dual(const void* q, const void* k, const void* v, const void* meta_buf,
+                      int batch, int total_tokens, int max_seqlen,
+                      int Hq, int Hkv, int head_dim, float softmax_scale,
+                      void* out_student, float* lse_student, void* out_teacher, float* lse_teacher,
+                      kvs_stream_t stream);
+
 /* Bytes needed for the backward workspace (row sums, fp32 dQ accumulator, status). */
 size_t kvs_attn_bwd_workspace_bytes(int total_tokens, int Hq, int Hkv, int head_dim, int grad_dtype);
 
 /*
- * Backward of the same operation (gradients of sum(out * dout)):
+ * Backward of the same operation (Sec. 2, "KV-streams" paragraph: the trainer trains on that one trace,
+ * so the same mask governs the gradients; gradients of sum(out * dout)):
  *   D_i = dout_i.out_i;  P_ij = exp(S_ij - lse_i);  dP_ij = dout_i.v_j;  dS_ij = P_ij (dP_ij - D_i)
  *   dq_i = scale sum_j dS_ij k_j;  dk_j = scale sum_{h in group} sum_i dS_ij q_i;
  *   dv_j = sum_{h in group} sum_i P_ij dout_i
@@ -227,7 +246,9 @@ int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t* cu_seqlen
  * Eviction removes whole pages from a table and returns them to the stack; the rows never move.
  * Decode attention reads exactly the pages a table names; it never sees a mask.  Device-side
  * failures (cache full, a range that is not whole pages) set the status word, read with
- * kvs_cache_status().
+ * kvs_cache_status().  num_pages is the size of the cache: a table or stack entry outside
+ * [0, num_pages) is never followed; it is recorded as KVS_ERR_INVALID_ARG (in the cache status word by
+ * append/evict, in the workspace status word by decode attention, which then reads page 0 instead).
  * ---------------------------------------------------------------------------------------------- */
 size_t kvs_cache_free_list_bytes(int num_pages);
 /* All pages free, status OK. */
@@ -235,13 +256,13 @@ int kvs_cache_init(int32_t* free_list, int num_pages, kvs_stream_t stream);
 /* Appends one token (k_new, v_new: bf16 [num_seqs, Hkv, head_dim]) to every sequence whose `active`
  * byte is non-zero (active == NULL: all), taking a page from the stack when the last one is full. */
 int kvs_cache_append(const void* k_new, const void* v_new, const uint8_t* active,
-                     int num_seqs, int Hkv, int head_dim, int page_size, int max_pages,
+                     int num_seqs, int Hkv, int head_dim, int page_size, int max_pages, int num_pages,
                      int32_t* block_table, int32_t* n_tokens, int32_t* free_list,
                      void* k_cache, void* v_cache, kvs_stream_t stream);
 /* Physical eviction.  ranges: int32 [n_ranges, 3] rows (sequence, first_page_slot, n_pages) in
  * positions of the CURRENT table; the named table entries are removed (the rest keep their order),
  * n_tokens drops by n_pages * page_size, the pages go back on the stack. */
-int kvs_cache_evict(const int32_t* ranges, int n_ranges, int num_seqs, int page_size, int max_pages,
+int kvs_cache_evict(const int32_t* ranges, int n_ranges, int num_seqs, int page_size, int max_pages, int num_pages,
                     int32_t* block_table, int32_t* n_tokens, int32_t* free_list, kvs_stream_t stream);
 /* Reads the cache status word.  SYNCHRONISES the stream. */
 int kvs_cache_status(const int32_t* free_list, int* free_pages_host, kvs_stream_t stream);
@@ -259,7 +280,7 @@ size_t kvs_decode_workspace_bytes(int num_seqs, int Hq, int head_dim, int num_sp
  */
 int kvs_decode_attn(const void* q, const void* k_cache, const void* v_cache,
                     const int32_t* block_table, const int32_t* n_tokens,
-                    int num_seqs, int Hq, int Hkv, int head_dim, int page_size, int max_pages,
+                    int num_seqs, int Hq, int Hkv, int head_dim, int page_size, int max_pages, int num_pages,
                     float softmax_scale, int num_splits, void* out, float* lse,
                     void* workspace, size_t workspace_bytes, kvs_stream_t stream);
 

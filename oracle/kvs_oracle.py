@@ -413,3 +413,165 @@ class PagedCacheModel:
         self.tables[s] = kept
         self.free.extend(freed)
         self.n_tokens[s] -= len(freed) * self.page_size
+
+
+# --------------------------------------------------------------------------
+# operand rounding: what the 2e-2 / 5e-3 tolerances have to absorb
+# --------------------------------------------------------------------------
+# The method computes with bf16 operands and fp32 accumulation.  Apart from the inputs (already
+# bf16) three intermediate quantities are rounded to bf16 before they are used again: the
+# probabilities P (operand of P V and of P^T dO), the score gradients dS (operand of dS K and
+# dS^T Q) and the stored output O (which the row sums D = dO . O are formed from).  Two functions
+# state the consequence in fp64:
+#   dense_fwd_bwd_rounded   the definition with exactly those three roundings switched on or off;
+#                           with all of them off it is dense_fwd / dense_bwd, bit for bit
+#   rounding_sigma          first-order propagation of those roundings, as a standard deviation
+#                           per output element, treating every rounding error as independent with
+#                           the rms relative size RHO_BF16
+# The tests use them to bound the CUDA path's max-abs error element by element: 2e-2 wherever six
+# standard deviations of the inherent rounding stay below it, six standard deviations elsewhere.
+U_BF16 = 2.0 ** -8            # largest relative error of round-to-nearest to 8 significant bits
+# rms relative error of that rounding for significands spread log-uniformly over [1, 2):
+# sqrt(E[1/m^2] / 3) * 2^-8 with E[1/m^2] = (1/2 - 1/8) / ln 2
+RHO_BF16 = U_BF16 * float(np.sqrt((0.5 - 0.125) / np.log(2.0) / 3.0))
+
+
+def round_bf16(x):
+    """Nearest bf16 value (ties to even) of every element, returned as fp64."""
+    x32 = np.ascontiguousarray(np.asarray(x, dtype=np.float64).astype(np.float32))
+    bits = x32.view(np.uint32).astype(np.uint64)
+    bits = (bits + 0x7FFF + ((bits >> 16) & 1)) & 0xFFFF0000
+    return bits.astype(np.uint32).view(np.float32).reshape(x32.shape).astype(np.float64)
+
+
+def dense_fwd_bwd_rounded(q, k, v, dout, evict_at, scale, round_p=True, round_ds=True, round_out=True):
+    """dense_fwd + dense_bwd with the method's three operand roundings (see above).
+    Returns out, lse, dq, dk, dv (fp64; out holds bf16 values when round_out)."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    dout = np.asarray(dout, dtype=np.float64)
+    T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    check_evict_at(evict_at)
+    A = allowed(evict_at)
+    out = np.zeros((T, Hq, d))
+    lse = np.zeros((Hq, T))
+    dq = np.zeros_like(q)
+    dk = np.zeros_like(k)
+    dv = np.zeros_like(v)
+    for h in range(Hq):
+        g = h // G
+        S = scale * (q[:, h, :] @ k[:, g, :].T)
+        S = np.where(A, S, -np.inf)
+        m = S.max(axis=1, keepdims=True)
+        E = np.exp(S - m)
+        l = E.sum(axis=1, keepdims=True)       # the row sum is taken before the rounding
+        P = E / l
+        Pv = round_bf16(E) / l if round_p else P
+        O = Pv @ v[:, g, :]
+        if round_out:
+            O = round_bf16(O)
+        out[:, h, :] = O
+        lse[h, :] = (m + np.log(l))[:, 0]
+        Pb = round_bf16(P) if round_p else P
+        dP = dout[:, h, :] @ v[:, g, :].T
+        D = (dout[:, h, :] * O).sum(axis=1, keepdims=True)
+        dS = P * (dP - D)
+        if round_ds:
+            dSs = round_bf16(scale * dS)       # the scale is folded in before the rounding
+            dq[:, h, :] = dSs @ k[:, g, :]
+            dk[:, g, :] += dSs.T @ q[:, h, :]
+        else:
+            dq[:, h, :] = scale * (dS @ k[:, g, :])
+            dk[:, g, :] += scale * (dS.T @ q[:, h, :])
+        dv[:, g, :] += Pb.T @ dout[:, h, :]
+    return out, lse, dq, dk, dv
+
+
+def rounding_sigma(q, k, v, dout, evict_at, scale):
+    """Standard deviation, per element of out, dq, dk, dv, of the error that the three operand
+    roundings cause, to first order, every rounding error independent with relative rms RHO_BF16
+    (the output rounding of O: uniform within half a bf16 ulp of O).
+
+        out_ic:  P_ij e_ij v_jc summed over j, plus its own rounding
+        D_i   :  sum_c dO_ic (error of the stored O_ic); common to the whole row i of dS
+        dv_jc :  sum_{h,i} P_ij e_ij dO_ic
+        dq_ic :  s sum_j dS_ij e'_ij k_jc  -  s dD_i sum_j P_ij k_jc
+        dk_jc :  s sum_{h,i} (dS_ij e'_ij - P_ij dD_i) q_ic
+
+    Returns a dict of fp64 arrays shaped like the tensors."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    dout = np.asarray(dout, dtype=np.float64)
+    T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    A = allowed(evict_at)
+    r2 = RHO_BF16 ** 2
+    var_out = np.zeros((T, Hq, d))
+    var_dq = np.zeros_like(q)
+    var_dk = np.zeros_like(k)
+    var_dv = np.zeros_like(v)
+    for h in range(Hq):
+        g = h // G
+        kk, vv, qq, do = k[:, g, :], v[:, g, :], q[:, h, :], dout[:, h, :]
+        S = np.where(A, scale * (qq @ kk.T), -np.inf)
+        E = np.exp(S - S.max(axis=1, keepdims=True))
+        P = E / E.sum(axis=1, keepdims=True)
+        O = P @ vv
+        P2 = P * P
+        var_o_p = r2 * (P2 @ (vv * vv))                              # from the rounding of P
+        ulp_half = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(O), 1e-300))) - 8)
+        var_o = var_o_p + ulp_half ** 2 / 3.0                         # plus the rounding of O itself
+        var_out[:, h, :] = var_o
+        var_D = ((do * do) * var_o).sum(axis=1, keepdims=True)       # [T, 1]
+        dS = P * (do @ vv.T - (do * O).sum(axis=1, keepdims=True))
+        dS2 = dS * dS
+        var_dv[:, g, :] += r2 * (P2.T @ (do * do))
+        var_dq[:, h, :] = scale ** 2 * (r2 * (dS2 @ (kk * kk)) + var_D * (P @ kk) ** 2)
+        var_dk[:, g, :] += scale ** 2 * (r2 * (dS2.T @ (qq * qq)) + (P2 * var_D).T @ (qq * qq))
+    return {"out": np.sqrt(var_out), "dq": np.sqrt(var_dq), "dk": np.sqrt(var_dk), "dv": np.sqrt(var_dv)}
+
+
+def varlen_rounding_sigma(q, k, v, dout, evict_at, cu_seqlens, scale):
+    """rounding_sigma trace by trace over a packed batch."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    res = {"out": np.zeros_like(q), "dq": np.zeros_like(q), "dk": np.zeros_like(k), "dv": np.zeros_like(k)}
+    for b in range(len(cu_seqlens) - 1):
+        a, e = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        if e == a:
+            continue
+        s = rounding_sigma(q[a:e], k[a:e], v[a:e], dout[a:e], evict_at[a:e], scale)
+        for name in res:
+            res[name][a:e] = s[name]
+    return res
+
+
+# --------------------------------------------------------------------------
+# student + teacher forward (self-distillation, App. D.3 "Training Objectives")
+# --------------------------------------------------------------------------
+def dual_fwd(q, k, v, evict_at, scale):
+    """The two passes of the self-distillation objective on one trace, same q, k, v: the student under
+    the eviction mask, the teacher with the full causal context (nothing evicted).  By definition two
+    calls of dense_fwd.  Returns (out_student, lse_student, out_teacher, lse_teacher)."""
+    T = np.asarray(evict_at).shape[0]
+    os_, ls_ = dense_fwd(q, k, v, evict_at, scale)
+    ot_, lt_ = dense_fwd(q, k, v, np.full(T, INF, dtype=np.int64), scale)
+    return os_, ls_, ot_, lt_
+
+
+def varlen_dual_fwd(q, k, v, evict_at, cu_seqlens, scale):
+    q = np.asarray(q, dtype=np.float64)
+    Ttot, Hq, d = q.shape
+    res = [np.zeros((Ttot, Hq, d)), np.zeros((Hq, Ttot)), np.zeros((Ttot, Hq, d)), np.zeros((Hq, Ttot))]
+    for b in range(len(cu_seqlens) - 1):
+        a, e = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        if e == a:
+            continue
+        r = dual_fwd(q[a:e], k[a:e], v[a:e], evict_at[a:e], scale)
+        res[0][a:e], res[1][:, a:e], res[2][a:e], res[3][:, a:e] = r
+    return tuple(res)

@@ -38,6 +38,7 @@ SIGNATURES = {
     "kvs_mask_meta": (_i, [_vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "kvs_mask_meta_export": (_i, [_vp, _i, _vp, _i, _i, _vp, _vp, _vp, _vp]),
     "kvs_attn_fwd": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp]),
+    "kvs_attn_fwd_dual": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp]),
     "kvs_attn_bwd_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
     "kvs_attn_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "kvs_attn_bwd_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp,
@@ -48,12 +49,12 @@ SIGNATURES = {
     "kvs_selftest_bounded_wait": (_i, [_vp, _i, ctypes.c_longlong, _vp]),
     "kvs_cache_free_list_bytes": (_sz, [_i]),
     "kvs_cache_init": (_i, [_vp, _i, _vp]),
-    "kvs_cache_append": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
-    "kvs_cache_evict": (_i, [_vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
+    "kvs_cache_append": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "kvs_cache_evict": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "kvs_cache_status": (_i, [_vp, ctypes.POINTER(ctypes.c_int), _vp]),
     "kvs_decode_num_splits": (_i, [_i, _i, _i]),
     "kvs_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
-    "kvs_decode_attn": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _sz, _vp]),
+    "kvs_decode_attn": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _sz, _vp]),
     "kvs_host_arena_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "kvs_attn_fwd_bwd_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i,
                                    _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -72,7 +73,7 @@ def load() -> ctypes.CDLL:
     """Loads libkvs.so (built by paper_2609_35750_b200.build).  Raises if absent."""
     global _lib
     if _lib is None:
-        path = os.environ.get("KVS_LIB", LIB_PATH)       # KVS_LIB: an alternative build of the same library
+        path = LIB_PATH
         if not os.path.exists(path):
             raise FileNotFoundError(
                 f"{path} not found: build it with `python -m paper_2609_35750_b200.build`; there is no fallback path")
@@ -172,6 +173,29 @@ def kvs_attn_fwd(q, k, v, meta_buf, batch: int, max_seqlen: int, softmax_scale: 
                                float(softmax_scale), _dev(out, "out", torch.bfloat16), _dev(lse, "lse", torch.float32),
                                _stream(stream)), "kvs_attn_fwd")
     return out, lse
+
+
+def kvs_attn_fwd_dual(q, k, v, meta_buf, batch: int, max_seqlen: int, softmax_scale: float = 0.0,
+                      out_student=None, lse_student=None, out_teacher=None, lse_teacher=None, stream=None):
+    """Student (eviction mask) and teacher (full causal context) forward sharing every q k^T tile.
+    Returns (out_student, lse_student, out_teacher, lse_teacher)."""
+    total, Hq, d = q.shape
+    Hkv = k.shape[1]
+    if out_student is None:
+        out_student = torch.empty_like(q)
+    if out_teacher is None:
+        out_teacher = torch.empty_like(q)
+    if lse_student is None:
+        lse_student = torch.empty((Hq, total), dtype=torch.float32, device=q.device)
+    if lse_teacher is None:
+        lse_teacher = torch.empty((Hq, total), dtype=torch.float32, device=q.device)
+    _check(load().kvs_attn_fwd_dual(_dev(q, "q", torch.bfloat16), _dev(k, "k", torch.bfloat16), _dev(v, "v", torch.bfloat16),
+                                    _dev(meta_buf, "meta_buf", torch.uint8), batch, total, max_seqlen, Hq, Hkv, d,
+                                    float(softmax_scale), _dev(out_student, "out_student", torch.bfloat16),
+                                    _dev(lse_student, "lse_student", torch.float32),
+                                    _dev(out_teacher, "out_teacher", torch.bfloat16),
+                                    _dev(lse_teacher, "lse_teacher", torch.float32), _stream(stream)), "kvs_attn_fwd_dual")
+    return out_student, lse_student, out_teacher, lse_teacher
 
 
 def kvs_attn_bwd_workspace_bytes(total_tokens: int, Hq: int, Hkv: int, head_dim: int, grad_dtype: int) -> int:
@@ -298,7 +322,7 @@ class PagedCache:
     def append(self, k_new: torch.Tensor, v_new: torch.Tensor, active: Optional[torch.Tensor] = None, stream=None) -> None:
         _check(load().kvs_cache_append(_dev(k_new, "k_new", torch.bfloat16), _dev(v_new, "v_new", torch.bfloat16),
                                        _dev(active, "active", torch.uint8) if active is not None else None,
-                                       self.num_seqs, self.Hkv, self.d, self.page_size, self.max_pages,
+                                       self.num_seqs, self.Hkv, self.d, self.page_size, self.max_pages, self.num_pages,
                                        self.block_table.data_ptr(), self.n_tokens.data_ptr(), self.free_list.data_ptr(),
                                        self.k_cache.data_ptr(), self.v_cache.data_ptr(), _stream(stream)), "kvs_cache_append")
 
@@ -306,7 +330,7 @@ class PagedCache:
         """ranges int32 [n, 3] rows (sequence, first_page_slot, n_pages) (device)."""
         n = ranges.shape[0] if ranges.numel() else 0
         _check(load().kvs_cache_evict(_dev(ranges, "ranges", torch.int32) if n else None, n, self.num_seqs, self.page_size,
-                                      self.max_pages, self.block_table.data_ptr(), self.n_tokens.data_ptr(),
+                                      self.max_pages, self.num_pages, self.block_table.data_ptr(), self.n_tokens.data_ptr(),
                                       self.free_list.data_ptr(), _stream(stream)), "kvs_cache_evict")
 
     def status(self, stream=None) -> Tuple[int, int]:
@@ -330,7 +354,7 @@ class PagedCache:
             lse = torch.empty((S, Hq), dtype=torch.float32, device=q.device)
         _check(load().kvs_decode_attn(_dev(q, "q", torch.bfloat16), self.k_cache.data_ptr(), self.v_cache.data_ptr(),
                                       self.block_table.data_ptr(), self.n_tokens.data_ptr(), S, Hq, self.Hkv, d, self.page_size,
-                                      self.max_pages, float(softmax_scale), num_splits, _dev(out, "out", torch.bfloat16),
+                                      self.max_pages, self.num_pages, float(softmax_scale), num_splits, _dev(out, "out", torch.bfloat16),
                                       _dev(lse, "lse", torch.float32), _dev(workspace, "workspace", torch.uint8),
                                       workspace.numel(), _stream(stream)), "kvs_decode_attn")
         return out, lse

@@ -11,15 +11,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;   // looked up once; the driver entry point never changes
-    if (!fn) {
+    // looked up once (thread-safe static initialisation); the driver entry point never changes
+    static const EncodeTiledFn fn = []() -> EncodeTiledFn {
         void* ptr = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
             qres != cudaDriverEntryPointSuccess)
             return nullptr;
-        fn = (EncodeTiledFn)ptr;
-    }
+        return (EncodeTiledFn)ptr;
+    }();
     return fn;
 }
 

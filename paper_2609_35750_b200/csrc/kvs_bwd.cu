@@ -132,7 +132,8 @@ struct BwdSmem {
 };
 
 struct BwdParams {
-    int total_tokens, Hq, Hkv;
+    int batch, total_tokens, max_seqlen;   // what the caller says meta_buf was built for
+    int Hq, Hkv;
     float scale, scale_log2;
     const float* lse;
     const float* dvec;
@@ -141,14 +142,6 @@ struct BwdParams {
     int grad_fp32;
     int32_t* status;
 };
-
-#ifdef KVS_TRACE
-// Debug build only: clock64 timestamps of one CTA's pipeline events.
-__device__ long long g_trace[8192];
-#define KVS_TR(slot, j, ev) do { if ((j) >= 8 && (j) < 20) s_tr[((j) - 8) * 16 + (ev)] = (uint32_t)clock64(); } while (0)
-#else
-#define KVS_TR(slot, j, ev) do { } while (0)
-#endif
 
 template <int D>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
@@ -169,6 +162,11 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
+    // meta_buf must be the one kvs_mask_meta wrote for these sizes: every index below comes out of it
+    if (!meta_matches(mv.hdr, p.batch, p.total_tokens, p.max_seqlen)) {
+        if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) set_status(p.status, KVS_ERR_BAD_META);
+        return;
+    }
     if ((int)blockIdx.x >= mv.hdr->nblk_total) return;
     const int gb = mv.bwd_order[blockIdx.x];
     const int g = blockIdx.y;
@@ -193,9 +191,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const uint32_t sK = sbase + L::OFF_K, sV = sbase + L::OFF_V, sQ = sbase + L::OFF_Q, sDO = sbase + L::OFF_DO,
                    sDS = sbase + L::OFF_DS, sSTG = sbase + L::OFF_STG;
     uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(sgen + L::OFF_MISC);
-#ifdef KVS_TRACE
-    volatile uint32_t* s_tr = reinterpret_cast<volatile uint32_t*>(sgen + L::TOTAL);   // 12 iterations x 16 events
-#endif
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + L::OFF_MISC + 4);
     const uint32_t bars = sbase + L::OFF_BAR;
     const uint32_t bar_kv = bars;
@@ -302,28 +297,23 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 const uint32_t ph = j & 1;
                 const uint64_t so = s ? STAGE : 0;
                 // dP^T(j) = V dO^T  (its columns hold dQ(j-1) until the drain warps have read it)
-                KVS_TR(0, j, 2);
                 mbar_wait(bar_dofull, ph, abort_flag, status);
                 if (j > 0) mbar_wait(bar_drained, (j - 1) & 1, abort_flag, status);
                 tc_fence_after();
-                KVS_TR(0, j, 3);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
                     if (leader) mma_ss(tmem_P, dV_k + off, dDO_k + off, IDESC_ST, kk > 0);
                 }
                 if (leader) mma_commit(bar_dp);
-                KVS_TR(0, j, 4);
                 // dV(j) += P^T dO
                 mbar_wait(bar_p, ph, abort_flag, status);
                 tc_fence_after();
-                KVS_TR(0, j, 1);
 #pragma unroll
                 for (int kk = 0; kk < TILE / 16; ++kk)
                     if (leader) mma_ts(tmem_dV, tmem_S + (kk >> 2) * 64 + (kk & 3) * 8, dDO_mn + (uint64_t)(kk * 128), IDESC_KV,
                            (j > 0) || (kk > 0));
                 if (leader) mma_commit(bar_dofree);
-                KVS_TR(0, j, 5);
                 // S^T(j+1) = K Q^T
                 if (j + 1 < n_iter) {
                     const uint64_t so1 = s ? 0 : STAGE;
@@ -341,7 +331,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 // K-major A operand of dK; dQ goes first so that the drain can start while dK still runs.
                 mbar_wait(bar_dss, ph, abort_flag, status);
                 tc_fence_after();
-                KVS_TR(0, j, 6);
 #pragma unroll
                 for (int kk = 0; kk < TILE / 16; ++kk)
                     if (leader) mma_ss(tmem_P, dDS_mn + (uint64_t)(kk * 128), dK_mn + (uint64_t)(kk * 128), IDESC_DQ, kk > 0);
@@ -352,7 +341,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     if (leader) mma_ss(tmem_dK, dDS_k + off, dQ_mn + so + (uint64_t)(kk * 128), IDESC_KV, (j > 0) || (kk > 0));
                 }
                 if (leader) mma_commit(bar_qfree(s));
-                KVS_TR(0, j, 7);
             }
         }
     } else if (warp >= 8) {
@@ -367,7 +355,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const int m = n + j % nm;
             mbar_wait(bar_dq, j & 1, abort_flag, status);
             tc_fence_after();
-            if (tid == 256) KVS_TR(1, j, 8);
             uint32_t r[D];
 #pragma unroll
             for (int ch = 0; ch < D / 32; ++ch) {
@@ -380,7 +367,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_drained);      // the columns may be overwritten from here on
-            if (tid == 256) KVS_TR(1, j, 9);
             // chunks of 32 head-dim columns through two staging buffers
 #pragma unroll
             for (int ch = 0; ch < D / 32; ++ch) {
@@ -426,7 +412,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             mbar_wait(bar_ldfull(s), (j >> 1) & 1, abort_flag, status);
             mbar_wait(bar_s, j & 1, abort_flag, status);
             tc_fence_after();
-            if (tid == 0) KVS_TR(2, j, 10);
             const float4* l4 = reinterpret_cast<const float4*>(sLse + s * TILE + col0);
             uint32_t r0[32], r1[32];
             tmem_ld32(tmem_S + lane_sel + col0, r0);
@@ -459,20 +444,17 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_p);
-            if (tid == 0) KVS_TR(2, j, 11);
         };
 
         auto phase_ds = [&](int j) {       // dS^T(j) = P^T (scale dP^T - scale D)
             const int s = j & 1;
             mbar_wait(bar_dp, j & 1, abort_flag, status);
             tc_fence_after();
-            if (tid == 0) KVS_TR(2, j, 12);
             const float4* d4 = reinterpret_cast<const float4*>(sDv + s * TILE + col0);
             uint32_t r0[32], r1[32];
             tmem_ld32(tmem_P + lane_sel + col0, r0);
             tmem_ld32(tmem_P + lane_sel + col0 + 32, r1);
             tmem_wait_ld();
-            if (tid == 0) KVS_TR(2, j, 14);
             uint32_t dk_[32];
             const float2 sc2 = make_float2(p.scale, p.scale);
 #pragma unroll
@@ -492,12 +474,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             for (int c = 0; c < 8; ++c)
                 *reinterpret_cast<uint4*>(sDS_row + ((c ^ (row & 7)) << 4)) =
                     make_uint4(dk_[c * 4], dk_[c * 4 + 1], dk_[c * 4 + 2], dk_[c * 4 + 3]);
-            if (tid == 0) KVS_TR(2, j, 15);
             fence_proxy_async();                     // dS visible to the tensor core's reads of shared memory
             tc_fence_before();                       // orders this thread's reads of dP^T before the dQ MMA that overwrites it
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_dss);
-            if (tid == 0) KVS_TR(2, j, 13);
         };
 
         phase_p(0);
@@ -545,9 +525,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
     tc_fence_before();
     __syncthreads();
-#ifdef KVS_TRACE
-    if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 192) g_trace[tid] = s_tr[tid];
-#endif
     if (warp == 13) {
         __syncwarp();
         tmem_dealloc(tmem, TMEM_COLS);
@@ -617,7 +594,9 @@ extern "C" int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, c
     char* ws = (char*)workspace;
     const size_t nq = (size_t)total_tokens * Hq * head_dim;
     BwdParams p;
+    p.batch = batch;
     p.total_tokens = total_tokens;
+    p.max_seqlen = max_seqlen < total_tokens ? max_seqlen : total_tokens;
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.scale = softmax_scale == 0.f ? 1.0f / sqrtf((float)head_dim) : softmax_scale;
@@ -653,8 +632,3 @@ extern "C" int kvs_attn_bwd(const void* dout, const void* q, const void* k, cons
                            grad_dtype, dq, dk, dv, workspace, workspace_bytes, stream, nullptr, nullptr);
 }
 
-#ifdef KVS_TRACE
-extern "C" int kvs_debug_read_trace(long long* host, int n) {
-    return cudaMemcpyFromSymbol(host, kvs::g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : -1;
-}
-#endif

@@ -125,6 +125,15 @@ int check_device_sm100();
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void set_status(int32_t* status, int code) { atomicCAS(status, 0, code); }
 
+// True when `hdr` is the header kvs_mask_meta wrote for exactly these sizes (max_seqlen already
+// clamped to total_tokens, as kvs_mask_meta stores it).  The attention kernels test this before
+// they read any index out of the buffer: a buffer built for other sizes has its arrays at other
+// offsets, and one that was never built holds arbitrary indices.
+__device__ __forceinline__ bool meta_matches(const MetaHeader* hdr, int batch, int total_tokens, int max_seqlen) {
+    return hdr->magic == META_MAGIC && hdr->batch == batch && hdr->total_tokens == total_tokens &&
+           hdr->max_seqlen == max_seqlen;
+}
+
 // ------------------------------------------------------------------------------------------
 // device: PTX wrappers (sm_100a)
 // ------------------------------------------------------------------------------------------

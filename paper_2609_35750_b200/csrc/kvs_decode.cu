@@ -31,11 +31,20 @@ struct DecodeParams {
     const __nv_bfloat16* v_cache;
     const int32_t* block_table;      // [S, max_pages]
     const int32_t* n_tokens;         // [S]
-    int S, Hq, Hkv, page_size, max_pages, nsplit;
+    int S, Hq, Hkv, page_size, max_pages, num_pages, nsplit;
+    int32_t* status;                 // workspace status word: a page id outside [0, num_pages) is recorded there
     float scale_log2;
     float* part_o;                   // [S, Hq, nsplit, D] unnormalised
     float* part_ml;                  // [S, Hq, nsplit, 2]  (max in base-2 units, sum)
 };
+
+// A block-table entry is only followed if it names a page of the cache: anything else (a stale or
+// corrupt table) is recorded as KVS_ERR_INVALID_ARG and read as page 0, so no kernel reads outside the cache.
+__device__ __forceinline__ int checked_page(const DecodeParams& p, int page) {
+    if ((unsigned)page < (unsigned)p.num_pages) return page;
+    set_status(p.status, KVS_ERR_INVALID_ARG);
+    return 0;
+}
 
 // 16 bytes (CH = 8) or 8 bytes (CH = 4) of a bf16 row, widened to fp32
 template <int CH>
@@ -68,7 +77,7 @@ decode_partial_kernel(DecodeParams p) {
     const int z = blockIdx.x, g = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int half = lane >> 4, l16 = lane & 15;
-    const int n = p.n_tokens[s];
+    const int n = min(max(p.n_tokens[s], 0), p.max_pages * p.page_size);    // never past the sequence's table
     const int ps = p.page_size;
     const int nblocks = (n + BLK - 1) / BLK;
     // blocks of this split, dealt round-robin to (split, warp)
@@ -102,7 +111,7 @@ decode_partial_kernel(DecodeParams p) {
         // row index (page * page_size + offset) of token t0 + l16, fetched once per block by every lane;
         // tokens past the end are clamped to the last one (their scores are discarded below)
         const int tl = min(t0 + (l16 & (BLK - 1)), n - 1);
-        const int my_row = bt[tl / ps] * ps + tl % ps;
+        const int my_row = checked_page(p, bt[tl / ps]) * ps + tl % ps;
         // ---- all K rows of the block in flight, then the scores ----
         RowChunk<CH> raw[ROWS];
         int rowi[ROWS];
@@ -250,7 +259,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     const int z = blockIdx.x, g = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n = p.n_tokens[s];
+    const int n = min(max(p.n_tokens[s], 0), p.max_pages * p.page_size);    // never past the sequence's table
     const int ps = p.page_size;
     const int ppt = 128 / ps;                                   // pages per tile
     const int ntiles = (n + 127) >> 7;
@@ -315,7 +324,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             if (PAGED_TMA && leader) {
                 mbar_expect_tx(bar_full, (uint32_t)(npages * ps) * 512u);
                 for (int i = 0; i < npages; ++i) {
-                    const int row = bt[tt * ppt + i] * ps;
+                    const int row = checked_page(p, bt[tt * ppt + i]) * ps;
                     const uint32_t off = (uint32_t)(i * ps) * 128u;
                     tma_load_3d(sK + off, &tm_k, 0, g, row, bar_full);
                     tma_load_3d(sK + BOX + off, &tm_k, 64, g, row, bar_full);
@@ -363,7 +372,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             for (int j = 0; j < 16; ++j) {
                 const int r = warp * 32 + 2 * j + (lane >> 4);
                 const int tok = tt * 128 + r;
-                nrow[j] = (r < nvalid) ? (long long)bt[tok / ps] * ps + tok % ps : -1;
+                nrow[j] = (r < nvalid) ? (long long)checked_page(p, bt[tok / ps]) * ps + tok % ps : -1;
             }
         };
         auto load_tile_rows = [&]() {
@@ -551,7 +560,7 @@ __global__ void cache_init_kernel(int32_t* free_buf, int num_pages) {
 // one thread per sequence: take a page when the last one is full, write the token's K and V rows
 __global__ void cache_append_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
                                     const uint8_t* __restrict__ active, int S, int Hkv, int D, int page_size, int max_pages,
-                                    int32_t* block_table, int32_t* n_tokens, int32_t* free_buf, __nv_bfloat16* k_cache,
+                                    int num_pages, int32_t* block_table, int32_t* n_tokens, int32_t* free_buf, __nv_bfloat16* k_cache,
                                     __nv_bfloat16* v_cache) {
     CacheHeader* hdr = reinterpret_cast<CacheHeader*>(free_buf);
     int32_t* stack = free_buf + 4;
@@ -566,9 +575,9 @@ __global__ void cache_append_kernel(const __nv_bfloat16* __restrict__ k_new, con
                 atomicCAS(&hdr->status, 0, KVS_ERR_WORKSPACE);
             } else {
                 const int top = atomicSub(&hdr->top, 1);
-                if (top <= 0) {
+                if (top <= 0 || top > num_pages) {
                     atomicAdd(&hdr->top, 1);
-                    atomicCAS(&hdr->status, 0, KVS_ERR_WORKSPACE);       // cache full
+                    atomicCAS(&hdr->status, 0, top <= 0 ? KVS_ERR_WORKSPACE : KVS_ERR_INVALID_ARG);   // cache full / corrupt stack
                 } else {
                     page = stack[top - 1];
                     block_table[(size_t)s * max_pages + slot / page_size] = page;
@@ -576,6 +585,10 @@ __global__ void cache_append_kernel(const __nv_bfloat16* __restrict__ k_new, con
             }
         } else {
             page = block_table[(size_t)s * max_pages + slot / page_size];
+        }
+        if (page >= num_pages || (page < 0 && page != -1)) {       // an entry that names no page of this cache
+            atomicCAS(&hdr->status, 0, KVS_ERR_INVALID_ARG);
+            page = -1;
         }
         s_page = page;
     }
@@ -595,7 +608,7 @@ __global__ void cache_append_kernel(const __nv_bfloat16* __restrict__ k_new, con
 // one CTA per sequence: remove the pages [first_page, first_page + n_pages) of every listed range from the
 // block table (stable compaction of the table; the rows never move) and push them on the free list
 __global__ void cache_evict_kernel(const int32_t* __restrict__ ranges, int n_ranges, int S, int page_size, int max_pages,
-                                   int32_t* block_table, int32_t* n_tokens, int32_t* free_buf) {
+                                   int num_pages, int32_t* block_table, int32_t* n_tokens, int32_t* free_buf) {
     CacheHeader* hdr = reinterpret_cast<CacheHeader*>(free_buf);
     int32_t* stack = free_buf + 4;
     const int s = blockIdx.x;
@@ -605,8 +618,13 @@ __global__ void cache_evict_kernel(const int32_t* __restrict__ ranges, int n_ran
     const int n = n_tokens[s];
     const int npages = (n + page_size - 1) / page_size;
     int32_t* bt = block_table + (size_t)s * max_pages;
+    if (threadIdx.x == 0) s_bad = (n < 0 || npages > max_pages) ? 1 : 0;
+    __syncthreads();
+    if (s_bad) {
+        if (threadIdx.x == 0) atomicCAS(&hdr->status, 0, KVS_ERR_INVALID_ARG);
+        return;
+    }
     for (int i = threadIdx.x; i < npages; i += blockDim.x) sh[i] = 1;
-    if (threadIdx.x == 0) s_bad = 0;
     __syncthreads();
     for (int r = 0; r < n_ranges; ++r) {
         if (ranges[3 * r] != s) continue;
@@ -633,9 +651,17 @@ __global__ void cache_evict_kernel(const int32_t* __restrict__ ranges, int n_ran
             const unsigned gone = __ballot_sync(0xffffffffu, i < npages && sh[i] == 0);
             freed += __popc(gone);
         }
-        if (lane == 0) s_base = atomicAdd(&hdr->top, freed);
+        if (lane == 0) {
+            s_base = atomicAdd(&hdr->top, freed);
+            if (s_base < 0 || s_base + freed > num_pages) {        // more pages coming back than the cache has: corrupt state
+                atomicSub(&hdr->top, freed);
+                atomicCAS(&hdr->status, 0, KVS_ERR_INVALID_ARG);
+                s_base = -1;
+            }
+        }
         __syncwarp();
         const int base = s_base;
+        if (base < 0) return;
         int fpos = 0;
         for (int i0 = 0; i0 < npages; i0 += 32) {
             const int i = i0 + lane;
@@ -682,21 +708,22 @@ extern "C" int kvs_cache_status(const int32_t* free_list, int* free_pages_host, 
 }
 
 extern "C" int kvs_cache_append(const void* k_new, const void* v_new, const uint8_t* active, int num_seqs, int Hkv, int head_dim,
-                                int page_size, int max_pages, int32_t* block_table, int32_t* n_tokens, int32_t* free_list,
+                                int page_size, int max_pages, int num_pages, int32_t* block_table, int32_t* n_tokens, int32_t* free_list,
                                 void* k_cache, void* v_cache, kvs_stream_t stream) {
     if (!k_new || !v_new || !block_table || !n_tokens || !free_list || !k_cache || !v_cache) return KVS_ERR_INVALID_ARG;
-    if (num_seqs < 0 || Hkv <= 0 || head_dim <= 0 || page_size <= 0 || max_pages <= 0) return KVS_ERR_INVALID_ARG;
+    if (num_seqs < 0 || Hkv <= 0 || head_dim <= 0 || page_size <= 0 || max_pages <= 0 || num_pages <= 0) return KVS_ERR_INVALID_ARG;
     if (num_seqs == 0) return KVS_OK;
     cache_append_kernel<<<num_seqs, 128, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, active,
-                                                                   num_seqs, Hkv, head_dim, page_size, max_pages, block_table,
+                                                                   num_seqs, Hkv, head_dim, page_size, max_pages, num_pages, block_table,
                                                                    n_tokens, free_list, (__nv_bfloat16*)k_cache,
                                                                    (__nv_bfloat16*)v_cache);
     return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
 }
 
-extern "C" int kvs_cache_evict(const int32_t* ranges, int n_ranges, int num_seqs, int page_size, int max_pages, int32_t* block_table,
+extern "C" int kvs_cache_evict(const int32_t* ranges, int n_ranges, int num_seqs, int page_size, int max_pages, int num_pages,
+                               int32_t* block_table,
                                int32_t* n_tokens, int32_t* free_list, kvs_stream_t stream) {
-    if (!block_table || !n_tokens || !free_list || n_ranges < 0 || num_seqs < 0 || page_size <= 0 || max_pages <= 0)
+    if (!block_table || !n_tokens || !free_list || n_ranges < 0 || num_seqs < 0 || page_size <= 0 || max_pages <= 0 || num_pages <= 0)
         return KVS_ERR_INVALID_ARG;
     if (n_ranges > 0 && !ranges) return KVS_ERR_INVALID_ARG;
     if ((size_t)max_pages * sizeof(int32_t) > 200 * 1024) return KVS_ERR_UNSUPPORTED;
@@ -705,7 +732,7 @@ extern "C" int kvs_cache_evict(const int32_t* ranges, int n_ranges, int num_seqs
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(cache_evict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return KVS_ERR_CUDA;
-    cache_evict_kernel<<<num_seqs, 256, smem, (cudaStream_t)stream>>>(ranges, n_ranges, num_seqs, page_size, max_pages, block_table,
+    cache_evict_kernel<<<num_seqs, 256, smem, (cudaStream_t)stream>>>(ranges, n_ranges, num_seqs, page_size, max_pages, num_pages, block_table,
                                                                      n_tokens, free_list);
     return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
 }
@@ -761,10 +788,11 @@ static int launch_decode(const DecodeParams& p, int G, const void* k_cache, cons
         memset(&tk, 0, sizeof(tk));
         memset(&tv, 0, sizeof(tv));
         if (paged_tma) {
-            // the caches as (d, Hkv, rows) with rows = pages * page_size; the row count is not known here, and the
-            // map only uses it to clip boxes, which never stick out (a box is one page)
-            if ((rc = make_tmap_thd(&tk, k_cache, 1 << 30, p.Hkv, 128, ps)) != KVS_OK) return rc;
-            if ((rc = make_tmap_thd(&tv, v_cache, 1 << 30, p.Hkv, 128, ps)) != KVS_OK) return rc;
+            // the caches as (d, Hkv, rows) with rows = num_pages * page_size: a box is one page, and no box
+            // can reach past the cache (the table entries are range-checked on top of that)
+            if ((long long)p.num_pages * ps > 0x7fffffffLL) return KVS_ERR_UNSUPPORTED;
+            if ((rc = make_tmap_thd(&tk, k_cache, p.num_pages * ps, p.Hkv, 128, ps)) != KVS_OK) return rc;
+            if ((rc = make_tmap_thd(&tv, v_cache, p.num_pages * ps, p.Hkv, 128, ps)) != KVS_OK) return rc;
             switch (G) {
                 case 1: rc = launch_decode_tc<1, true>(tk, tv, p, status, st); break;
                 case 2: rc = launch_decode_tc<2, true>(tk, tv, p, status, st); break;
@@ -798,9 +826,10 @@ static int launch_decode(const DecodeParams& p, int G, const void* k_cache, cons
 
 extern "C" int kvs_decode_attn(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_table,
                                const int32_t* n_tokens, int num_seqs, int Hq, int Hkv, int head_dim, int page_size, int max_pages,
-                               float softmax_scale, int num_splits, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                               int num_pages, float softmax_scale, int num_splits, void* out, float* lse, void* workspace, size_t workspace_bytes,
                                kvs_stream_t stream) {
-    if (num_seqs < 0 || Hq <= 0 || Hkv <= 0 || page_size <= 0 || max_pages <= 0 || num_splits <= 0) return KVS_ERR_INVALID_ARG;
+    if (num_seqs < 0 || Hq <= 0 || Hkv <= 0 || page_size <= 0 || max_pages <= 0 || num_pages <= 0 || num_splits <= 0)
+        return KVS_ERR_INVALID_ARG;
     if (head_dim != 64 && head_dim != 128) return KVS_ERR_UNSUPPORTED;
     if (Hq % Hkv != 0 || num_seqs > 65535 || Hkv > 65535) return KVS_ERR_UNSUPPORTED;
     if (num_seqs == 0) return KVS_OK;
@@ -820,6 +849,8 @@ extern "C" int kvs_decode_attn(const void* q, const void* k_cache, const void* v
     p.Hkv = Hkv;
     p.page_size = page_size;
     p.max_pages = max_pages;
+    p.num_pages = num_pages;
+    p.status = (int32_t*)workspace + 1;
     p.nsplit = num_splits;
     const float s = softmax_scale == 0.f ? 1.0f / sqrtf((float)head_dim) : softmax_scale;
     p.scale_log2 = s * 1.4426950408889634f;

@@ -39,23 +39,17 @@ struct FwdSmem {
     static constexpr int OFF_BAR = OFF_FLAG + 16;
     static constexpr int OFF_MISC = OFF_BAR + 24 * 8;
     static constexpr int TOTAL = OFF_MISC + 16;
-    static constexpr int DYN_BYTES = TOTAL + 1024 + 1024;   // slack for the 1024-byte alignment (+ room for a debug trace)
+    static constexpr int DYN_BYTES = TOTAL + 1024;          // slack for the 1024-byte alignment
 };
 
 struct FwdParams {
-    int total_tokens, Hq, Hkv;
+    int batch, total_tokens, max_seqlen;   // what the caller says meta_buf was built for
+    int Hq, Hkv;
     float scale_log2;   // softmax_scale * log2(e)
     __nv_bfloat16* out;
     float* lse;
 };
 
-#ifdef KVS_TRACE
-// Debug build only: clock64 timestamps of one CTA's pipeline events.
-__device__ long long g_trace_fwd[1024];
-#define KVS_TRF(i, ev) do { if ((i) >= 8 && (i) < 20) s_tr[((i) - 8) * 16 + (ev)] = (uint32_t)clock64(); } while (0)
-#else
-#define KVS_TRF(i, ev) do { } while (0)
-#endif
 
 template <int D>
 __global__ void __launch_bounds__(FWD_THREADS, 1)
@@ -73,6 +67,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
+    // meta_buf must be the one kvs_mask_meta wrote for these sizes: every index below comes out of it
+    if (!meta_matches(mv.hdr, p.batch, p.total_tokens, p.max_seqlen)) {
+        if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) set_status(&mv.hdr->status, KVS_ERR_BAD_META);
+        return;
+    }
     if ((int)blockIdx.x >= mv.hdr->nblk_total) return;
     const int gb = mv.fwd_order[blockIdx.x];
     const int G = p.Hq / p.Hkv;
@@ -101,9 +100,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     volatile int32_t* sFlag = reinterpret_cast<volatile int32_t*>(sgen + L::OFF_FLAG);
     uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(sgen + L::OFF_MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + L::OFF_MISC + 4);
-#ifdef KVS_TRACE
-    volatile uint32_t* s_tr = reinterpret_cast<volatile uint32_t*>(sgen + L::TOTAL);
-#endif
     const uint32_t bars = sbase + L::OFF_BAR;
     const uint32_t bar_q = bars;
     auto bar_vfull = [&](int s) { return bars + 8 * (1 + s); };     // TMA bytes of V
@@ -254,34 +250,27 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     //                   B = V, MN-major, 16 key rows per step
                     // The first P_SPLIT keys of P arrive while the row's last exponentials are still being
                     // taken, so most of this product overlaps the tail of the softmax.
-                    KVS_TRF(i, t * 4 + 0);
                     mbar_wait(bar_p0(t), i & 1, abort_flag, status);
                     if (t == 0) mbar_wait(bar_vfull(s), (i >> 1) & 1, abort_flag, status);
                     tc_fence_after();
-                    KVS_TRF(i, t * 4 + 1);
 #pragma unroll
                     for (int kk = 0; kk < P_SPLIT / 16; ++kk)
                         if (leader) mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, dV0 + s * 2 * TBU + (uint64_t)(kk * 128), IDESC_O,
                                (i > 0) || (kk > 0));
-                    if (t == 0) KVS_TRF(i, 9);
                     mbar_wait(bar_p(t), i & 1, abort_flag, status);
                     tc_fence_after();
-                    if (t == 0) KVS_TRF(i, 10);
 #pragma unroll
                     for (int kk = P_SPLIT / 16; kk < TILE / 16; ++kk)
                         if (leader) mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, dV0 + s * 2 * TBU + (uint64_t)(kk * 128), IDESC_O, true);
                     if (leader && t == ntile - 1) mma_commit(bar_vfree(s));       // V(i) is not read by anything issued later
                     if (i + 1 < nlist) {
-                        KVS_TRF(i, t * 4 + 3);
                         if (t == 0) {
                             mbar_wait(bar_kfull(s ^ 1), ((i + 1) >> 1) & 1, abort_flag, status);
                             tc_fence_after();
-                            KVS_TRF(i, 15);
                         }
                         issue_s(t, s ^ 1);
                         if (leader && t == ntile - 1) mma_commit(bar_kfree(s ^ 1));
                     }
-                    KVS_TRF(i, t * 4 + 2);
                 }
             }
             if (leader) mma_commit(bar_done);
@@ -310,8 +299,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 const bool need_mask = sFlag[s] != 0;
                 mbar_wait(bar_s(t), it & 1, abort_flag, status);
                 tc_fence_after();
-                if (tid == 0) KVS_TRF(i, 8);
-                if (tid == 128) KVS_TRF(i, 13);
                 // raw logits of this row (the softmax scale is positive, so the maximum can be taken before it)
                 float sv[TILE];
                 {
@@ -419,8 +406,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p(t));
-                if (t == 0 && tid == 0) KVS_TRF(i, 12);
-                if (tid == 128) KVS_TRF(i, 14);
             }
 
             // ---- epilogue: O / l -> bf16, LSE -> fp32 ----
@@ -499,9 +484,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     if (nlist == 0 && tid == 0) mbar_wait(bar_q, 0, abort_flag, status);
     tc_fence_before();
     __syncthreads();
-#ifdef KVS_TRACE
-    if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 192) g_trace_fwd[tid] = s_tr[tid];
-#endif
     if (warp == 9) {
         __syncwarp();
         tmem_dealloc(tmem, TMEM_COLS);
@@ -543,7 +525,9 @@ extern "C" int kvs_attn_fwd(const void* q, const void* k, const void* v, const v
     if ((rc = make_tmap_thd(&tk, k, total_tokens, Hkv, head_dim, TILE)) != KVS_OK) return rc;
     if ((rc = make_tmap_thd(&tv, v, total_tokens, Hkv, head_dim, TILE)) != KVS_OK) return rc;
     FwdParams p;
+    p.batch = batch;
     p.total_tokens = total_tokens;
+    p.max_seqlen = max_seqlen < total_tokens ? max_seqlen : total_tokens;
     p.Hq = Hq;
     p.Hkv = Hkv;
     const float s = softmax_scale == 0.f ? 1.0f / sqrtf((float)head_dim) : softmax_scale;
@@ -554,8 +538,3 @@ extern "C" int kvs_attn_fwd(const void* q, const void* k, const void* v, const v
     return head_dim == 64 ? launch_fwd<64>(tq, tk, tv, mv, p, L.nb_cap, st) : launch_fwd<128>(tq, tk, tv, mv, p, L.nb_cap, st);
 }
 
-#ifdef KVS_TRACE
-extern "C" int kvs_debug_read_trace_fwd(long long* host, int n) {
-    return cudaMemcpyFromSymbol(host, kvs::g_trace_fwd, sizeof(long long) * n) == cudaSuccess ? 0 : -1;
-}
-#endif

@@ -90,3 +90,32 @@ def shard_workload(w, rank: int, world_size: int):
     sub = Workload(f"{w.name}[rank{rank}/{world_size}]", cu, ev.astype(np.int32), w.Hq, w.Hkv, w.d,
                    q_prescale=w.q_prescale, softmax_scale=w.softmax_scale, notes=w.notes)
     return sub, idx.astype(np.int64)
+
+
+def spawn_local(n: int, argv: Sequence[str], env_extra=None, master_port: int = 0, timeout=None) -> List[Tuple[int, str]]:
+    """Starts `n` local ranks of the command `argv` (one process per GPU: RANK = LOCAL_RANK = 0..n-1,
+    WORLD_SIZE = n, rendezvous on 127.0.0.1) and waits for all of them.  Returns [(exit code, stdout text)]
+    by rank; stderr passes through.  If one rank fails the others are left to their process-group timeout
+    or are terminated once `timeout` seconds have passed."""
+    import socket
+    import subprocess
+    if master_port <= 0:
+        s = socket.socket()
+        s.bind(("127.0.0.1", 0))
+        master_port = s.getsockname()[1]
+        s.close()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ)
+        env.update(env_extra or {})
+        env.update(RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(master_port))
+        procs.append(subprocess.Popen(list(argv), env=env, stdout=subprocess.PIPE, text=True))
+    results: List[Tuple[int, str]] = []
+    for p in procs:
+        try:
+            out, _ = p.communicate(timeout=timeout)
+        except subprocess.TimeoutExpired:
+            p.kill()
+            out, _ = p.communicate()
+        results.append((p.returncode, out or ""))
+    return results

@@ -2,10 +2,11 @@
 batches of ragged traces, four mask families.  Every case runs mask metadata, forward and backward through the
 C ABI and compares all five outputs.
 
-Bounds: relative L2 5e-3 as everywhere.  The absolute bound 2e-2 is stated for the named configs; here group size and
-trace length are arbitrary, and a gradient that sums bf16-rounded P or dS terms (2^-9 relative each) over G heads and up
-to 1400 queries reaches |dv| ~ 10, so the absolute bound is max(2e-2, 2^-8 * max|reference|) (seen: 0.0202 on a
-G = 7 case with |dv| up to 9)."""
+Bounds: relative L2 5e-3 as everywhere.  The absolute bound 2e-2 is stated for the named configs; here group size,
+trace length and mask are arbitrary.  P and dS are rounded to bf16 (relative rms 1.66e-3) before they are summed into
+dv, dk, dq over the G heads of a group and over every query that sees a key, so the first keys of a trace, which every
+query sees with a large probability, collect the most noise.  The oracle propagates those roundings to a standard
+deviation per element (oracle.rounding_sigma); an element's bound is max(2e-2, six of its standard deviations)."""
 import numpy as np
 import pytest
 import torch
@@ -54,12 +55,13 @@ def test_random_shapes_match_the_oracle(seed):
         assert B.kvs_device_status(meta) == B.KVS_OK
         ro, rl = O.varlen_fwd(f(q), f(k), f(v), w.evict_at, w.cu_seqlens, w.scale)
         rdq, rdk, rdv = O.varlen_bwd(f(q), f(k), f(v), f(do), w.evict_at, w.cu_seqlens, w.scale)
+        sg = O.varlen_rounding_sigma(f(q), f(k), f(v), f(do), w.evict_at, w.cu_seqlens, w.scale)
         what = dict(Hq=w.Hq, Hkv=w.Hkv, d=w.d, lens=np.diff(w.cu_seqlens).tolist())
         for name, got, ref in (("out", out, ro), ("lse", lse, rl), ("dq", dq, rdq), ("dk", dk, rdk), ("dv", dv, rdv)):
             g = f(got)
             assert np.isfinite(g).all(), (name, what)
-            bound = max(2e-2, 2.0 ** -8 * float(np.abs(ref).max()))
-            assert np.abs(g - ref).max() <= bound, (name, what, float(np.abs(g - ref).max()), bound)
+            bound = np.maximum(2e-2, 6.0 * sg[name]) if name in sg and name != "out" else 2e-2
+            assert (np.abs(g - ref) <= bound).all(), (name, what, float(np.abs(g - ref).max()))
             nref = np.linalg.norm(ref)
             if nref > 1e-3:
                 assert np.linalg.norm(g - ref) / nref <= 5e-3, (name, what)

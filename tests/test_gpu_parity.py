@@ -5,7 +5,11 @@ product of each pair, which alone gives about 2e-3 relative L2):
     max |gpu - oracle| <= 2e-2   and   ||gpu - oracle||_2 / ||oracle||_2 <= 5e-3
 for out, lse and, with fp32 gradient outputs, dq, dk, dv.  With bf16 gradient outputs the
 max-abs bound is 2e-2 or one bf16 ulp of the oracle value, whichever is larger (a value of
-magnitude 8..16 cannot be stored in bf16 more finely than 0.03).  Mask metadata is bit-exact.
+magnitude 8..16 cannot be stored in bf16 more finely than 0.03).  Where a case leaves the value
+range or group width of the five configurations, the max-abs bound of an element is instead
+max(2e-2, six standard deviations of the method's own operand rounding at that element), the
+deviation coming from the oracle's first-order model (oracle.rounding_sigma), never from a measured
+error.  The relative bound is the same everywhere.  Mask metadata is bit-exact.
 """
 import numpy as np
 import pytest
@@ -22,19 +26,25 @@ REL_L2 = 5e-3
 DEV = "cuda"
 
 
-def _close(name, got, ref, bf16_out=False, max_abs=None):
-    MAX_ABS = max_abs if max_abs is not None else globals()["MAX_ABS"]
+def _close(name, got, ref, bf16_out=False, sigma=None):
+    """max-abs and relative-L2 check of one tensor.  sigma (optional, shaped like ref): the oracle's
+    per-element standard deviation of the method's own operand rounding (oracle.rounding_sigma); where
+    six of them exceed 2e-2 the element's bound is six of them, elsewhere it stays 2e-2."""
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (name, got.shape, ref.shape)
     assert np.isfinite(got).all(), f"{name}: non-finite values"
     err = np.abs(got - ref)
+    bound = np.full(ref.shape, MAX_ABS)
+    if sigma is not None:
+        bound = np.maximum(bound, 6.0 * sigma)
     if bf16_out:
         ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(ref), 1e-30))) - 7)
-        bound = np.maximum(MAX_ABS, ulp)
-        assert (err <= bound).all(), f"{name}: max-abs {err.max():.4f} beyond max(2e-2, 1 bf16 ulp)"
-    else:
-        assert err.max() <= MAX_ABS, f"{name}: max-abs {err.max():.4f} > {MAX_ABS}"
+        # a bf16 result carries up to half an ulp of its own rounding on top of the computation's error;
+        # without a noise model the element's bound is one ulp where that is more than 2e-2
+        bound = np.maximum(bound, ulp) if sigma is None else np.maximum(MAX_ABS, 6.0 * sigma + 0.5 * ulp)
+    worst = np.unravel_index(np.argmax(err - bound), err.shape)
+    assert (err <= bound).all(), f"{name}: |error| {err[worst]:.4f} at {worst} beyond its bound {bound[worst]:.4f}"
     if np.linalg.norm(ref) > 1e-3:      # a reference that is identically zero has no relative error
         rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
         assert rel <= REL_L2, f"{name}: rel-L2 {rel:.3e} > {REL_L2}"
@@ -65,7 +75,9 @@ def _check_meta(w, meta):
     assert np.array_equal(kmax, np.concatenate([b for _, b in mm]))
 
 
-def _full_parity(w, seed=0, tensors=None, bwd=True, dq_abs=None, dkv_abs=None):
+def _full_parity(w, seed=0, tensors=None, bwd=True, derived=False):
+    """derived=True: the max-abs bound of the gradients follows the oracle's rounding model element by
+    element (for inputs outside the configs' value range or group width); otherwise it is 2e-2 flat."""
     q, k, v, do = tensors if tensors is not None else W.make_tensors(w, seed)
     qd, kd, vd, dod = (t.to(DEV) for t in (q, k, v, do))
     meta, out, lse, dq, dk, dv = _run_gpu(w, qd, kd, vd, dod, B.GRAD_FP32)
@@ -77,16 +89,17 @@ def _full_parity(w, seed=0, tensors=None, bwd=True, dq_abs=None, dkv_abs=None):
     if not bwd:
         return out, lse, dq, dk, dv
     rdq, rdk, rdv = O.varlen_bwd(qn, kn, vn, don, w.evict_at, w.cu_seqlens, w.scale)
-    _close("dq", _f64(dq), rdq, max_abs=dq_abs)
-    _close("dk", _f64(dk), rdk, max_abs=dkv_abs)
-    _close("dv", _f64(dv), rdv, max_abs=dkv_abs)
+    sg = O.varlen_rounding_sigma(qn, kn, vn, don, w.evict_at, w.cu_seqlens, w.scale) if derived else {}
+    _close("dq", _f64(dq), rdq, sigma=sg.get("dq"))
+    _close("dk", _f64(dk), rdk, sigma=sg.get("dk"))
+    _close("dv", _f64(dv), rdv, sigma=sg.get("dv"))
     # bf16 gradient outputs: same kernels plus the cast pass
     _, out2, lse2, dq2, dk2, dv2 = _run_gpu(w, qd, kd, vd, dod, B.GRAD_BF16)
     assert dq2.dtype == torch.bfloat16
     assert torch.equal(out, out2) and torch.equal(lse, lse2)       # forward is run-to-run identical
-    _close("dq(bf16)", _f64(dq2), rdq, bf16_out=True, max_abs=dq_abs)
-    _close("dk(bf16)", _f64(dk2), rdk, bf16_out=True, max_abs=dkv_abs)
-    _close("dv(bf16)", _f64(dv2), rdv, bf16_out=True, max_abs=dkv_abs)
+    _close("dq(bf16)", _f64(dq2), rdq, bf16_out=True, sigma=sg.get("dq"))
+    _close("dk(bf16)", _f64(dk2), rdk, bf16_out=True, sigma=sg.get("dk"))
+    _close("dv(bf16)", _f64(dv2), rdv, bf16_out=True, sigma=sg.get("dv"))
     return out, lse, dq, dk, dv
 
 
@@ -108,15 +121,11 @@ def test_cfg0_full():
     ("cfg6_G16", dict(cfg=6, shrink=32, Hq=16, Hkv=1, batch=1)),        # non-monotone evict_at, a wide group
 ])
 def test_shrunk_configs_full_tensor(name, kw):
-    # Variant B of config 1 folds 1/sqrt(d) into Q and runs with softmax_scale = 1, so dq = 1 * dS k is
-    # sqrt(d) times larger than with the default scale (|dq| reaches ~36) and the rounding of dS to bf16
-    # alone moves it by more than 2e-2; its absolute bound is scaled by sqrt(d), the relative one is not.
-    dq_abs = MAX_ABS * np.sqrt(128.0) if name == "cfg1B_scale1" else None
-    # dk and dv of a KV head sum the bf16-rounded P and dS of its G query heads: with G = 16, twice the widest group
-    # of the configs the 2e-2 bound is stated for, the rounding noise is sqrt(2) times larger (measured 0.0226); the
-    # relative bound stays as it is
-    dkv_abs = MAX_ABS * np.sqrt(2.0) if name == "cfg6_G16" else None
-    _full_parity(W.make_workload(seed=1, **kw), seed=1, dq_abs=dq_abs, dkv_abs=dkv_abs)
+    # The flat 2e-2 bound is the one stated for the five configurations.  Two cases leave their range:
+    # variant B of config 1 runs with softmax_scale = 1 (dq = 1 * dS k is sqrt(d) times larger, |dq| reaches
+    # ~36) and a group of 16 heads sums twice as many rounded terms into dk, dv as the widest configuration.
+    # For them the bound follows the oracle's model of the method's own operand rounding, element by element.
+    _full_parity(W.make_workload(seed=1, **kw), seed=1, derived=name in ("cfg1B_scale1", "cfg6_G16"))
 
 
 @pytest.mark.parametrize("seed", [0, 1, 2])
@@ -206,8 +215,8 @@ def test_growing_logits_change_the_maximum_in_every_tile():
     q[:, :, 0] = 1.0
     k[:, :, 0] = (k[:, :, 0].float() + torch.arange(T, dtype=torch.float32)[:, None] * 0.02).to(torch.bfloat16)
     # k now has a component of size up to 20, and dq is a k-weighted sum of dS (rounded to bf16 as an
-    # MMA operand): its values and its rounding error grow with max|k|, so its absolute bound is scaled
-    _full_parity(w, tensors=(q, k, v, do), dq_abs=3 * MAX_ABS)
+    # MMA operand): its rounding error grows with |k|, which the oracle's rounding model accounts for
+    _full_parity(w, tensors=(q, k, v, do), derived=True)
 
 
 def test_zero_query_live_counts_on_gpu():
@@ -321,3 +330,25 @@ def test_host_buffer_entry_point_matches_device_path(Hq, Hkv, grad):
     assert torch.equal(ho, out.cpu()) and torch.equal(hl, lse.cpu())
     assert torch.equal(hdk, dk.cpu()) and torch.equal(hdv, dv.cpu())
     assert torch.allclose(hdq.float(), dq.cpu().float(), atol=2e-2, rtol=2e-2)
+
+
+# ---- the error of the CUDA path is the method's own operand rounding -------------------------------
+@pytest.mark.parametrize("kw", [dict(cfg=0), dict(cfg=2, shrink=32, Hq=8, Hkv=2, batch=1), dict(cfg=4, shrink=64, Hq=8, Hkv=1)])
+def test_error_is_explained_by_the_operand_rounding_model(kw):
+    # The oracle states which three quantities the method rounds to bf16 (P, dS, the stored O) and
+    # propagates those roundings to a standard deviation per output element.  If the kernels add no error
+    # of their own, (gpu - oracle) / sigma has rms close to 1 and no element is far out; a missing term, a
+    # rounding in the wrong place or accumulation in reduced precision would show as a larger rms.
+    w = W.make_workload(seed=4, **kw)
+    q, k, v, do = W.make_tensors(w, 4)
+    _, out, lse, dq, dk, dv = _run_gpu(w, *(t.to(DEV) for t in (q, k, v, do)), B.GRAD_FP32)
+    qn, kn, vn, don = (_f64(t) for t in (q, k, v, do))
+    ro, rl = O.varlen_fwd(qn, kn, vn, w.evict_at, w.cu_seqlens, w.scale)
+    rdq, rdk, rdv = O.varlen_bwd(qn, kn, vn, don, w.evict_at, w.cu_seqlens, w.scale)
+    sg = O.varlen_rounding_sigma(qn, kn, vn, don, w.evict_at, w.cu_seqlens, w.scale)
+    for name, got, ref in (("out", out, ro), ("dq", dq, rdq), ("dk", dk, rdk), ("dv", dv, rdv)):
+        z = (_f64(got) - ref) / np.maximum(sg[name], 1e-30)
+        rms = float(np.sqrt((z ** 2).mean()))
+        print(f"{w.name} {name}: rms of error / predicted deviation = {rms:.3f}, largest {np.abs(z).max():.2f}")
+        assert rms <= 1.25, (name, rms)
+        assert np.abs(z).max() <= 7.0, (name, float(np.abs(z).max()))

@@ -30,12 +30,28 @@ def _both_ways(w, seed):
     dq = torch.empty(q.shape, dtype=torch.float32, device=DEV)
     dk = torch.empty(k.shape, dtype=torch.float32, device=DEV)
     dv = torch.empty(v.shape, dtype=torch.float32, device=DEV)
+    # One call first: the library's device image (which holds the fixed scratch array) becomes resident when its
+    # first kernel is loaded, and that one-time cost is not what is measured here.
+    B.kvs_attn_bwd_noalloc(do, q, k, v, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale, dq=dq, dk=dk, dv=dv)
     torch.cuda.synchronize()
-    before = torch.cuda.memory_allocated()
-    _, _, _, scratch = B.kvs_attn_bwd_noalloc(do, q, k, v, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale,
-                                              dq=dq, dk=dk, dv=dv)
+    dq.fill_(float("nan"))
+    dk.fill_(float("nan"))
+    dv.fill_(float("nan"))
     torch.cuda.synchronize()
-    assert torch.cuda.memory_allocated() == before
+    # Two counters: torch's own allocator, and the driver's count of free device memory, which any
+    # cudaMalloc / cudaMallocAsync inside the library would lower whoever made it.
+    # (The driver's figure is device-wide; should something else on the GPU move it, the measurement is repeated.)
+    for attempt in range(3):
+        before = torch.cuda.memory_allocated()
+        free_before = torch.cuda.mem_get_info()[0]
+        _, _, _, scratch = B.kvs_attn_bwd_noalloc(do, q, k, v, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale,
+                                                  dq=dq, dk=dk, dv=dv)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == before
+        if torch.cuda.mem_get_info()[0] == free_before:
+            break
+    else:
+        raise AssertionError("free device memory changed across kvs_attn_bwd_noalloc on three attempts")
     assert scratch != 0 and B.kvs_device_status_ptr(scratch) == B.KVS_OK
     # dk, dv are written in a fixed order: identical.  dq is summed with fp32 atomics: the order varies.
     assert torch.equal(dk, ref[1]) and torch.equal(dv, ref[2])

@@ -16,6 +16,7 @@ are timed for a few steps each and reported under `per_config` in the same line.
 Smaller runs for profilers and other paths, all through the same library calls:
     --shrink S [--hq H --hkv H --batch B]   a shrunk copy of the configuration
     --path meta                             the mask-metadata pass alone (large batches: its bandwidth)
+    --path dual                             student + teacher forward in one pass against two separate forwards
     --path decode [--seqs --live --page-size --hq --hkv --head-dim --splits]
                                             rollout side: decode attention over a fragmented paged cache
 """
@@ -220,9 +221,12 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-def time_train_steps(torch, B, W, w, seed, dev, steps, warmup, grad, barrier=None, sampler=None):
+def time_train_steps(torch, B, W, w, seed, dev, steps, warmup, grad, barrier=None, sampler=None, reorder=0):
     """Mask metadata + forward + backward, `warmup` untimed and `steps` timed steps on the current stream.
-    Returns a dict of per-phase mean times (ms), the total, and the device status."""
+    Returns a dict of per-phase mean times (ms), the total, and the device status.
+    reorder > 0: the token-level path.  Every step also sorts the keys of each window of `reorder` keys by eviction step
+    (kvs_reorder_keys), brings k and v into that slot order, builds the metadata for the slots, and returns dk, dv to token
+    order; all of it inside the timed step (counted under the metadata time)."""
     q, k, v, do = W.make_tensors(w, seed=seed, device=str(dev))
     ev = torch.from_numpy(w.evict_at).to(dev)
     cu = torch.from_numpy(w.cu_seqlens).to(dev)
@@ -233,6 +237,9 @@ def time_train_steps(torch, B, W, w, seed, dev, steps, warmup, grad, barrier=Non
     out = torch.empty_like(q)
     lse = torch.empty((Hq, Tt), dtype=torch.float32, device=dev)
     dq, dk, dv = (torch.empty(t.shape, dtype=gdt, device=dev) for t in (q, k, v))
+    if reorder:
+        perm, kf, ke = (torch.empty(Tt, dtype=torch.int32, device=dev) for _ in range(3))
+        kp, vp, dkp, dvp = torch.empty_like(k), torch.empty_like(v), torch.empty_like(dk), torch.empty_like(dv)
     stream = torch.cuda.current_stream()
     mk = lambda: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     ev_fwd, ev_bwd, ev_meta = mk(), mk(), mk()
@@ -243,15 +250,25 @@ def time_train_steps(torch, B, W, w, seed, dev, steps, warmup, grad, barrier=Non
     def step(i=None):
         if i is not None:
             ev_meta[i][0].record(stream)
-        B.kvs_mask_meta(ev, cu, w.max_seqlen, meta_buf=meta)
+        if reorder:
+            B.kvs_reorder_keys(ev, cu, w.max_seqlen, reorder, perm=perm, key_first=kf, key_evict=ke)
+            B.kvs_permute_rows(k, perm, kp)
+            B.kvs_permute_rows(v, perm, vp)
+            B.kvs_mask_meta_keys(kf, ke, cu, w.max_seqlen, meta_buf=meta)
+        else:
+            B.kvs_mask_meta(ev, cu, w.max_seqlen, meta_buf=meta)
+        kk, vv, dkk, dvv = (kp, vp, dkp, dvp) if reorder else (k, v, dk, dv)
         if i is not None:
             ev_meta[i][1].record(stream)
             ev_fwd[i][0].record(stream)
-        B.kvs_attn_fwd(q, k, v, meta, w.batch, w.max_seqlen, w.softmax_scale, out=out, lse=lse)
+        B.kvs_attn_fwd(q, kk, vv, meta, w.batch, w.max_seqlen, w.softmax_scale, out=out, lse=lse)
         if i is not None:
             ev_fwd[i][1].record(stream)
-        B.kvs_attn_bwd(do, q, k, v, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale, grad, dq=dq, dk=dk, dv=dv,
+        B.kvs_attn_bwd(do, q, kk, vv, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale, grad, dq=dq, dk=dkk, dv=dvv,
                        workspace=ws, main_events=(ev_bwd[i] if i is not None else None))
+        if reorder:
+            B.kvs_permute_rows(dkp, perm, dk, inverse=True)
+            B.kvs_permute_rows(dvp, perm, dv, inverse=True)
 
     for _ in range(max(warmup, 0)):
         step()
@@ -285,16 +302,17 @@ def time_train_steps(torch, B, W, w, seed, dev, steps, warmup, grad, barrier=Non
 def run_per_config(torch, B, W, dev, peaks, gpu_index):
     """The other configurations on the same clock as the headline: 1 warm-up + 3 timed steps each."""
     res = {}
-    for key, cfg, variant in (("0", 0, ""), ("1", 1, ""), ("3", 3, ""), ("4", 4, ""), ("4_control", 4, "control")):
+    for key, cfg, variant, reorder in (("0", 0, "", 0), ("1", 1, "", 0), ("3", 3, "", 0), ("4", 4, "", 0),
+                                       ("4_keys_reordered", 4, "", 4096), ("4_control", 4, "control", 0)):
         w = W.make_workload(cfg, seed=0, variant=variant)
         sampler = ClockSampler(gpu_index)
-        r = time_train_steps(torch, B, W, w, 0, dev, steps=3, warmup=1, grad=B.GRAD_BF16, sampler=sampler)
+        r = time_train_steps(torch, B, W, w, 0, dev, steps=3, warmup=1, grad=B.GRAD_BF16, sampler=sampler, reorder=reorder)
         r.pop("tensors")
         torch.cuda.empty_cache()
         ms = r["ms_total"] / 3
         tf = W.fwd_bwd_flops(w) / (ms * 1e-3) / 1e12
         res[key] = {"workload": w.name, "tokens": w.total_tokens, "unmasked_pairs": W.count_pairs(w), "steps": 3, "warmup": 1,
-                    "ms_per_step": ms, "effective_tflops": tf, "frac_of_burst_peak": tf / float(peaks["bf16_tflops"]),
+                    "reorder_window": reorder, "ms_per_step": ms, "effective_tflops": tf, "frac_of_burst_peak": tf / float(peaks["bf16_tflops"]),
                     "tokens_per_s": w.total_tokens / (ms * 1e-3), "ms_fwd": r["ms_fwd"], "ms_bwd_main": r["ms_bwd_main"],
                     "sm_mhz_median": (r["clocks"] or {}).get("sm_mhz"), "reasons": (r["clocks"] or {}).get("reasons")}
     return res
@@ -390,6 +408,61 @@ def run_decode(args):
         "dtype": "bf16", "data": "synthetic"}), flush=True)
 
 
+def run_dual(args):
+    """--path dual: the self-distillation forward (student under the eviction mask + full-context teacher, sharing
+    every q k^T tile) against the two single-stream forwards it replaces, on the same inputs."""
+    import torch
+    from paper_2609_35750_b200 import binding as B
+    from paper_2609_35750_b200 import workloads as W
+    dev = "cuda"
+    w = W.make_workload(args.config, seed=0, shrink=args.shrink, Hq=args.hq, Hkv=args.hkv, variant=args.variant, batch=args.batch)
+    q, k, v, _ = W.make_tensors(w, seed=0, device=dev, with_dout=False)
+    ev = torch.from_numpy(w.evict_at).to(dev)
+    cu = torch.from_numpy(w.cu_seqlens).to(dev)
+    meta = B.kvs_mask_meta(ev, cu, w.max_seqlen)
+    meta_c = B.kvs_mask_meta(torch.full_like(ev, int(W.INF)), cu, w.max_seqlen)
+    o = [torch.empty_like(q) for _ in range(2)]
+    l = [torch.empty((w.Hq, w.total_tokens), dtype=torch.float32, device=dev) for _ in range(2)]
+
+    def dual():
+        B.kvs_attn_fwd_dual(q, k, v, meta, w.batch, w.max_seqlen, w.softmax_scale, out_student=o[0], lse_student=l[0],
+                            out_teacher=o[1], lse_teacher=l[1])
+
+    def separate():
+        B.kvs_attn_fwd(q, k, v, meta, w.batch, w.max_seqlen, w.softmax_scale, out=o[0], lse=l[0])
+        B.kvs_attn_fwd(q, k, v, meta_c, w.batch, w.max_seqlen, w.softmax_scale, out=o[1], lse=l[1])
+
+    def timed(fn):
+        for _ in range(max(args.warmup, 1)):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    ms_dual, ms_sep = timed(dual), timed(separate)
+    if B.kvs_device_status(meta) != 0 or B.kvs_device_status(meta_c) != 0:
+        raise SystemExit("device status set")
+    pairs_s = W.count_pairs(w)
+    lens = np.diff(w.cu_seqlens).astype(np.int64)
+    pairs_t = int((lens * (lens + 1) // 2).sum())
+    flops = 4.0 * w.d * w.Hq * (pairs_s + pairs_t)        # what two separate forwards compute (unmasked pairs of both masks)
+    peaks = load_peaks()
+    tf = flops / (ms_dual * 1e-3) / 1e12
+    print(json.dumps({"metric": "dual_forward_effective_tflops", "value": tf, "unit": "TFLOP/s", "steps": args.steps, "warmup": args.warmup,
+                      "ms_per_step": ms_dual, "ms_two_separate_forwards": ms_sep, "speedup_over_separate": ms_sep / ms_dual,
+                      "config": {"workload": w.name, "tokens": w.total_tokens, "Hq": w.Hq, "Hkv": w.Hkv, "head_dim": w.d,
+                                 "student_pairs": pairs_s, "teacher_pairs": pairs_t,
+                                 "flops": "4*d*Hq*(student pairs + teacher pairs): the shared q k^T is counted once per stream"},
+                      "roofline": {"kernel": "fwd_dual_kernel", "bound": "tensor", "achieved": tf, "peak": float(peaks["bf16_tflops"]),
+                                   "unit": "TFLOP/s", "frac": tf / float(peaks["bf16_tflops"]), "traffic": None},
+                      "dtype": "bf16", "data": "synthetic"}), flush=True)
+
+
 def spawn_ranks(n):
     """`python bench.py --gpus N` without a launcher: start the N ranks here (one process per GPU, LOCAL_RANK = GPU
     index), pass rank 0's JSON line through, everything else the ranks print goes to stderr."""
@@ -420,7 +493,7 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="workload 0..7 (default 2: keep-last-4-turns, the target config)")
     ap.add_argument("--variant", type=str, default="")
     ap.add_argument("--impl", type=str, default="native", choices=["native", "reference"])
-    ap.add_argument("--path", type=str, default="train", choices=["train", "meta", "decode"])
+    ap.add_argument("--path", type=str, default="train", choices=["train", "meta", "decode", "dual"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-config", action="store_true")
@@ -430,6 +503,8 @@ def main():
     ap.add_argument("--hkv", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="number of traces (default: the configuration's own)")
     ap.add_argument("--grad", type=str, default="bf16", choices=["bf16", "fp32"])
+    ap.add_argument("--reorder", type=int, default=0,
+                    help="token-level eviction: sort the keys of every window of this many keys by eviction step (0: off)")
     ap.add_argument("--seqs", type=int, default=64, help="--path decode: sequences")
     ap.add_argument("--live", type=int, default=7168, help="--path decode: live tokens per sequence")
     ap.add_argument("--page-size", type=int, default=16, help="--path decode: tokens per page")
@@ -447,6 +522,9 @@ def main():
     if args.path == "decode":
         run_decode(args)
         return
+    if args.path == "dual":
+        run_dual(args)
+        return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         spawn_ranks(args.gpus)
         return
@@ -454,7 +532,7 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    small = args.shrink != 1 or args.hq is not None or args.hkv is not None or args.batch is not None
+    small = args.shrink != 1 or args.hq is not None or args.hkv is not None or args.batch is not None or args.reorder != 0
 
     # CPU baseline first (rank 0, N = 1 only), before this process touches CUDA
     cpu_baseline = None
@@ -479,7 +557,8 @@ def main():
     grad = B.GRAD_BF16 if args.grad == "bf16" else B.GRAD_FP32
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    r = time_train_steps(torch, B, W, w, rank, dev, args.steps, args.warmup, grad, barrier=D.barrier, sampler=sampler)
+    r = time_train_steps(torch, B, W, w, rank, dev, args.steps, args.warmup, grad, barrier=D.barrier, sampler=sampler,
+                         reorder=args.reorder)
     q, k, v, do = r.pop("tensors")
     clocks = r["clocks"]
     ms_total = r["ms_total"]
@@ -550,6 +629,7 @@ def main():
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "traces": w.batch, "tokens": Tt, "Hq": Hq, "Hkv": Hkv, "head_dim": d,
                    "unmasked_pairs": pairs, "flops_per_step": W.fwd_bwd_flops(w), "grad_dtype": args.grad,
+                   "reorder_window": args.reorder,
                    "l2": "inputs larger than L2 (q, dout, out, dq are each %.2f GB)" % (Tt * Hq * d * 2 / 1e9),
                    "parallelism": f"independent batches x{world}" if world > 1 else "single GPU", "notes": w.notes},
         "tokens_per_s": tokens_total / (ms_total_max * 1e-3),
@@ -566,7 +646,7 @@ def main():
                      "flops_per_launch": flops_bwd_main},
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": (8 if grad == B.GRAD_BF16 else 7) * args.steps,
+        "gpu_launches": ((8 if grad == B.GRAD_BF16 else 7) + (5 if args.reorder else 0)) * args.steps,
         "cpu_baseline": cpu_baseline,
         "per_config": per_config,
     }

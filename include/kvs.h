@@ -93,6 +93,44 @@ int kvs_mask_meta(const int32_t* evict_at, const int32_t* cu_seqlens,
                   void* meta_buf, size_t meta_bytes, kvs_stream_t stream);
 
 /*
+ * Mask metadata for key slots that carry their own visibility interval: slot j of a trace holds a key
+ * that query i of the trace may read iff  key_first[j] <= i < key_evict[j]  (both int32 [total_tokens],
+ * trace-local).  kvs_mask_meta is the case key_first[j] = j.  Two uses:
+ *   - token-level eviction (App. A.4): with the keys of a trace re-ordered by kvs_reorder_keys, the
+ *     slots of a 128-slot block die at about the same time, so most tiles are FULL or EMPTY instead of
+ *     PARTIAL; the attention calls then take k, v in the re-ordered slot order (kvs_permute_rows) and
+ *     return dk, dv in that order;
+ *   - any other visibility rule of this form, e.g. "visible from its eviction on" (key_first = evict_at,
+ *     key_evict = never), the complement of the eviction mask within the causal one.
+ * A slot may be visible to no query at all (key_first >= key_evict); a query row that sees no key gets
+ * out = 0 and lse = -inf.  Per block the classes use min/max of both arrays:
+ *     EMPTY if min key_first > q1 or q0 >= max key_evict;  FULL if max key_first <= q0 and q1 < min key_evict.
+ * kvs_attn_fwd_dual does not accept such a buffer (its status becomes KVS_ERR_UNSUPPORTED).
+ */
+int kvs_mask_meta_keys(const int32_t* key_first, const int32_t* key_evict, const int32_t* cu_seqlens,
+                       int batch, int total_tokens, int max_seqlen,
+                       void* meta_buf, size_t meta_bytes, kvs_stream_t stream);
+
+/*
+ * Key order for token-level eviction (App. A.4 "Turn-Wise Compaction" discusses token-level eviction):
+ * attention does not depend on the order of its keys, so the keys of a trace may be stored in any order
+ * as long as each carries its index and its eviction step.  Within every window of `window` consecutive
+ * keys of a trace (1 <= window <= 4096) the keys are sorted by (evict_at, index).  Outputs, all int32
+ * [total_tokens]: perm[s] = packed token index of the key that goes to slot s; key_first[s] = its
+ * trace-local index; key_evict[s] = its evict_at.  With turn-aligned evictions the order does not change.
+ */
+int kvs_reorder_keys(const int32_t* evict_at, const int32_t* cu_seqlens, int batch, int total_tokens, int max_seqlen,
+                     int window, int32_t* perm, int32_t* key_first, int32_t* key_evict, kvs_stream_t stream);
+
+/*
+ * Row permutation for tensors whose leading dimension is the packed token: rows of row_bytes bytes
+ * (a multiple of 16).  inverse == 0: dst row s = src row perm[s] (k, v into slot order);
+ * inverse != 0: dst row perm[s] = src row s (dk, dv back to token order).  src and dst must not overlap.
+ */
+int kvs_permute_rows(const void* src, const int32_t* perm, void* dst, long long n_rows, long long row_bytes,
+                     int inverse, kvs_stream_t stream);
+
+/*
  * Test/inspection hook: copies the classes and per-block min/max to HOST arrays and
  * SYNCHRONISES the stream.  tile_class_host: uint8, trace after trace, each trace a dense
  * row-major [nb x nb] matrix (nb = ceil(T_b/128); n > m is EMPTY).  kmin_host/kmax_host:

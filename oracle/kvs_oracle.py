@@ -45,13 +45,18 @@ EMPTY, PARTIAL, FULL = 0, 1, 2
 # --------------------------------------------------------------------------
 # mask
 # --------------------------------------------------------------------------
-def allowed(evict_at: np.ndarray) -> np.ndarray:
-    """Boolean [T, T]: allowed[i, j] = (j <= i) and (i < evict_at[j])."""
+def allowed(evict_at: np.ndarray, key_first=None) -> np.ndarray:
+    """Boolean [T, T]: allowed[i, j] = (j <= i) and (i < evict_at[j]).
+
+    With ``key_first`` (int [T]) column j is a key SLOT that carries its own interval: allowed[i, j] =
+    (key_first[j] <= i) and (i < evict_at[j]).  Attention does not depend on the order of its keys, so a
+    trace's keys may be stored in any order as long as slot j carries the index and the eviction step of
+    the key it holds; ``key_first[j] = j`` is the plain case."""
     ev = np.asarray(evict_at, dtype=np.int64)
     T = ev.shape[0]
     i = np.arange(T, dtype=np.int64)[:, None]
-    j = np.arange(T, dtype=np.int64)[None, :]
-    return (j <= i) & (i < ev[None, :])
+    first = np.arange(T, dtype=np.int64) if key_first is None else np.asarray(key_first, dtype=np.int64)
+    return (first[None, :] <= i) & (i < ev[None, :])
 
 
 def check_evict_at(evict_at: np.ndarray) -> None:
@@ -65,17 +70,20 @@ def check_evict_at(evict_at: np.ndarray) -> None:
 # --------------------------------------------------------------------------
 # dense masked attention, one trace
 # --------------------------------------------------------------------------
-def dense_fwd(q, k, v, evict_at, scale):
+def dense_fwd(q, k, v, evict_at, scale, key_first=None):
     """q [T,Hq,d], k,v [T,Hkv,d] (any float dtype; widened to fp64).
-    Returns out [T,Hq,d] fp64, lse [Hq,T] fp64 (natural log, scale included)."""
+    Returns out [T,Hq,d] fp64, lse [Hq,T] fp64 (natural log, scale included).
+    With ``key_first`` the rows of k, v are key slots (see ``allowed``); a query that sees no slot gets
+    out = 0 and lse = -inf."""
     q = np.asarray(q, dtype=np.float64)
     k = np.asarray(k, dtype=np.float64)
     v = np.asarray(v, dtype=np.float64)
     T, Hq, d = q.shape
     Hkv = k.shape[1]
     G = Hq // Hkv
-    check_evict_at(evict_at)
-    A = allowed(evict_at)
+    if key_first is None:
+        check_evict_at(evict_at)
+    A = allowed(evict_at, key_first)
     out = np.zeros((T, Hq, d))
     lse = np.zeros((Hq, T))
     for h in range(Hq):
@@ -83,17 +91,19 @@ def dense_fwd(q, k, v, evict_at, scale):
         S = scale * (q[:, h, :] @ k[:, g, :].T)
         S = np.where(A, S, -np.inf)
         m = S.max(axis=1, keepdims=True)
+        m = np.where(np.isfinite(m), m, 0.0)           # a row that sees nothing: every term below is zero
         E = np.exp(S - m)
         l = E.sum(axis=1, keepdims=True)
-        P = E / l
+        P = E / np.where(l > 0, l, 1.0)
         out[:, h, :] = P @ v[:, g, :]
-        lse[h, :] = (m + np.log(l))[:, 0]
+        with np.errstate(divide="ignore"):
+            lse[h, :] = (m + np.log(l))[:, 0]
     return out, lse
 
 
-def dense_bwd(q, k, v, dout, evict_at, scale):
+def dense_bwd(q, k, v, dout, evict_at, scale, key_first=None):
     """Analytic gradients of sum(out * dout) w.r.t. q, k, v.
-    Returns dq [T,Hq,d], dk, dv [T,Hkv,d] (fp64)."""
+    Returns dq [T,Hq,d], dk, dv [T,Hkv,d] (fp64).  ``key_first``: as in dense_fwd."""
     q = np.asarray(q, dtype=np.float64)
     k = np.asarray(k, dtype=np.float64)
     v = np.asarray(v, dtype=np.float64)
@@ -101,7 +111,7 @@ def dense_bwd(q, k, v, dout, evict_at, scale):
     T, Hq, d = q.shape
     Hkv = k.shape[1]
     G = Hq // Hkv
-    A = allowed(evict_at)
+    A = allowed(evict_at, key_first)
     dq = np.zeros_like(q)
     dk = np.zeros_like(k)
     dv = np.zeros_like(v)
@@ -110,8 +120,10 @@ def dense_bwd(q, k, v, dout, evict_at, scale):
         S = scale * (q[:, h, :] @ k[:, g, :].T)
         S = np.where(A, S, -np.inf)
         m = S.max(axis=1, keepdims=True)
+        m = np.where(np.isfinite(m), m, 0.0)
         E = np.exp(S - m)
-        P = E / E.sum(axis=1, keepdims=True)
+        l = E.sum(axis=1, keepdims=True)
+        P = E / np.where(l > 0, l, 1.0)
         O = P @ v[:, g, :]
         dP = dout[:, h, :] @ v[:, g, :].T
         D = (dout[:, h, :] * O).sum(axis=1, keepdims=True)
@@ -295,7 +307,7 @@ def key_block_dkdv(q, k, v, dout, evict_at, j0, j1, g, G, scale):
 # tile classes
 # --------------------------------------------------------------------------
 def block_minmax(evict_at, block=BLOCK):
-    """kmin[n], kmax[n] over the valid keys of key block n (one trace)."""
+    """kmin[n], kmax[n] over the valid keys (key slots) of key block n (one trace)."""
     ev = np.asarray(evict_at, dtype=np.int64)
     T = ev.shape[0]
     nb = (T + block - 1) // block
@@ -308,19 +320,25 @@ def block_minmax(evict_at, block=BLOCK):
     return kmin, kmax
 
 
-def tile_classes_rule(evict_at, block=BLOCK):
+def tile_classes_rule(evict_at, block=BLOCK, key_first=None):
     """Classes [nb, nb] uint8 from the min/max rule.  With q0, q1 the first and
     last valid query of block m and k0, k1 the first and last valid key of
     block n: EMPTY if k0 > q1 or q0 >= kmax[n]; FULL if k1 <= q0 and
-    q1 < kmin[n]; otherwise PARTIAL."""
+    q1 < kmin[n]; otherwise PARTIAL.  With ``key_first`` (key slots, see ``allowed``) k0 and k1 are
+    the smallest and the largest key_first of the block's slots."""
     T = len(evict_at)
     nb = (T + block - 1) // block
     kmin, kmax = block_minmax(evict_at, block)
+    if key_first is None:
+        fmin = np.arange(nb, dtype=np.int64) * block
+        fmax = np.minimum(fmin + block - 1, T - 1)
+    else:
+        fmin, fmax = block_minmax(key_first, block)
     cls = np.zeros((nb, nb), dtype=np.uint8)
     for m in range(nb):
         q0, q1 = m * block, min(m * block + block - 1, T - 1)
         for n in range(nb):
-            k0, k1 = n * block, min(n * block + block - 1, T - 1)
+            k0, k1 = int(fmin[n]), int(fmax[n])
             if k0 > q1 or q0 >= int(kmax[n]):
                 c = EMPTY
             elif k1 <= q0 and q1 < int(kmin[n]):
@@ -331,10 +349,10 @@ def tile_classes_rule(evict_at, block=BLOCK):
     return cls
 
 
-def tile_classes_brute(evict_at, block=BLOCK):
+def tile_classes_brute(evict_at, block=BLOCK, key_first=None):
     """Classes [nb, nb] uint8 straight from the boolean mask: all allowed ->
     FULL, none -> EMPTY, else PARTIAL."""
-    A = allowed(evict_at)
+    A = allowed(evict_at, key_first)
     T = A.shape[0]
     nb = (T + block - 1) // block
     cls = np.zeros((nb, nb), dtype=np.uint8)
@@ -575,3 +593,38 @@ def varlen_dual_fwd(q, k, v, evict_at, cu_seqlens, scale):
         r = dual_fwd(q[a:e], k[a:e], v[a:e], evict_at[a:e], scale)
         res[0][a:e], res[1][:, a:e], res[2][a:e], res[3][:, a:e] = r
     return tuple(res)
+
+
+# --------------------------------------------------------------------------
+# key order for token-level eviction; partial results over disjoint key sets
+# --------------------------------------------------------------------------
+def reorder_keys(evict_at, window):
+    """Permutation of one trace's keys: within every window of ``window`` consecutive keys, sorted by
+    (evict_at, index).  Returns perm (perm[s] = index of the key stored in slot s).  The slots then carry
+    key_first = perm and key_evict = evict_at[perm]; the attention result is unchanged (sums over keys do
+    not depend on their order), but the slots of a 128-slot block now leave the cache at about the same
+    time, which is what lets a tile be classified FULL or EMPTY (App. A.4 discusses token-level eviction)."""
+    ev = np.asarray(evict_at, dtype=np.int64)
+    T = ev.shape[0]
+    perm = np.zeros(T, dtype=np.int64)
+    for w0 in range(0, T, window):
+        idx = list(range(w0, min(w0 + window, T)))
+        idx.sort(key=lambda j: (int(ev[j]), j))
+        perm[w0:w0 + len(idx)] = idx
+    return perm
+
+
+def merge_partial(out_a, lse_a, out_b, lse_b):
+    """Attention over the union of two DISJOINT key sets from the results over each: with weights
+    w_x = exp(lse_x - lse), lse = log(exp(lse_a) + exp(lse_b)):  out = w_a out_a + w_b out_b.
+    out_* [T,Hq,d], lse_* [Hq,T]; a part that saw no key has lse = -inf and weight 0."""
+    la = np.asarray(lse_a, dtype=np.float64)
+    lb = np.asarray(lse_b, dtype=np.float64)
+    m = np.maximum(la, lb)
+    m0 = np.where(np.isfinite(m), m, 0.0)
+    with np.errstate(divide="ignore"):
+        lse = m0 + np.log(np.exp(la - m0) + np.exp(lb - m0))
+    wa = np.exp(la - np.where(np.isfinite(lse), lse, 0.0)) * np.isfinite(la)
+    wb = np.exp(lb - np.where(np.isfinite(lse), lse, 0.0)) * np.isfinite(lb)
+    out = wa.T[:, :, None] * np.asarray(out_a, dtype=np.float64) + wb.T[:, :, None] * np.asarray(out_b, dtype=np.float64)
+    return out, lse

@@ -36,6 +36,9 @@ SIGNATURES = {
     "kvs_mask_meta_bytes": (_sz, [_i, _i, _i]),
     "kvs_evict_at_from_events": (_i, [_vp, _i, _vp, _i, _i, _vp, _vp]),
     "kvs_mask_meta": (_i, [_vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "kvs_mask_meta_keys": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "kvs_reorder_keys": (_i, [_vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
+    "kvs_permute_rows": (_i, [_vp, _vp, _vp, ctypes.c_longlong, ctypes.c_longlong, _i, _vp]),
     "kvs_mask_meta_export": (_i, [_vp, _i, _vp, _i, _i, _vp, _vp, _vp, _vp]),
     "kvs_attn_fwd": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp]),
     "kvs_attn_fwd_dual": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp]),
@@ -142,6 +145,46 @@ def kvs_mask_meta(evict_at: torch.Tensor, cu_seqlens: torch.Tensor, max_seqlen: 
                                 batch, total, max_seqlen, _dev(meta_buf, "meta_buf", torch.uint8),
                                 meta_buf.numel(), _stream(stream)), "kvs_mask_meta")
     return meta_buf
+
+
+def kvs_mask_meta_keys(key_first: torch.Tensor, key_evict: torch.Tensor, cu_seqlens: torch.Tensor, max_seqlen: int,
+                       meta_buf: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Metadata for key slots with their own visibility interval [key_first, key_evict) (int32 [Ttot], device)."""
+    batch = cu_seqlens.numel() - 1
+    total = key_evict.numel()
+    if meta_buf is None:
+        meta_buf = torch.empty(kvs_mask_meta_bytes(batch, total, max_seqlen), dtype=torch.uint8, device=key_evict.device)
+    _check(load().kvs_mask_meta_keys(_dev(key_first, "key_first", torch.int32), _dev(key_evict, "key_evict", torch.int32),
+                                     _dev(cu_seqlens, "cu_seqlens", torch.int32), batch, total, max_seqlen,
+                                     _dev(meta_buf, "meta_buf", torch.uint8), meta_buf.numel(), _stream(stream)), "kvs_mask_meta_keys")
+    return meta_buf
+
+
+def kvs_reorder_keys(evict_at: torch.Tensor, cu_seqlens: torch.Tensor, max_seqlen: int, window: int, perm=None, key_first=None,
+                     key_evict=None, stream=None):
+    """Returns (perm, key_first, key_evict), int32 [Ttot] each: the keys of every trace sorted by (evict_at, index)
+    within windows of `window` keys."""
+    total = evict_at.numel()
+    mk = lambda t: t if t is not None else torch.empty(total, dtype=torch.int32, device=evict_at.device)
+    perm, key_first, key_evict = mk(perm), mk(key_first), mk(key_evict)
+    _check(load().kvs_reorder_keys(_dev(evict_at, "evict_at", torch.int32), _dev(cu_seqlens, "cu_seqlens", torch.int32),
+                                   cu_seqlens.numel() - 1, total, max_seqlen, window, _dev(perm, "perm", torch.int32),
+                                   _dev(key_first, "key_first", torch.int32), _dev(key_evict, "key_evict", torch.int32),
+                                   _stream(stream)), "kvs_reorder_keys")
+    return perm, key_first, key_evict
+
+
+def kvs_permute_rows(src: torch.Tensor, perm: torch.Tensor, dst: Optional[torch.Tensor] = None, inverse: bool = False, stream=None):
+    """dst[s] = src[perm[s]] (inverse False) or dst[perm[s]] = src[s] (inverse True) along the leading dimension."""
+    if dst is None:
+        dst = torch.empty_like(src)
+    n = src.shape[0]
+    row_bytes = (src.numel() // max(n, 1)) * src.element_size()
+    if not src.is_cuda or not src.is_contiguous() or not dst.is_contiguous() or dst.shape != src.shape or dst.dtype != src.dtype:
+        raise ValueError("src and dst must be contiguous CUDA tensors of the same shape and dtype")
+    _check(load().kvs_permute_rows(src.data_ptr(), _dev(perm, "perm", torch.int32), dst.data_ptr(), n, row_bytes, 1 if inverse else 0,
+                                   _stream(stream)), "kvs_permute_rows")
+    return dst
 
 
 def kvs_mask_meta_export(meta_buf: torch.Tensor, cu_seqlens_host, total_tokens: int, max_seqlen: int, stream=None):

@@ -176,10 +176,23 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const int tok0 = mv.seq_start[b];
     const int T = mv.seq_start[b + 1] - tok0;
     const int nb = (T + TILE - 1) / TILE;
+    const int m_first = mv.col_first[gb];           // == n unless the key slots were re-ordered
     const int m_last = mv.col_last[gb];
-    const int nm = m_last - n + 1;                  // query blocks n .. m_last see this key block
+    const int nm = m_last - m_first + 1;            // query blocks m_first .. m_last can see this key block
     const int n_iter = G * nm;
     int32_t* status = p.status;
+    const bool general = mv.hdr->general != 0;
+    if (nm <= 0) {
+        // no query sees any key of the block (general metadata only): its gradients are zero
+        const int rows = min(TILE, T - n * TILE);
+        const size_t per_row = (size_t)D * (p.grad_fp32 ? 4 : 2) / 16;          // 16-byte words of one (token, head) row
+        for (int i = tid; i < rows * (int)per_row; i += BWD_THREADS) {
+            const size_t off = ((size_t)(tok0 + n * TILE + i / (int)per_row) * p.Hkv + g) * per_row + i % (int)per_row;
+            reinterpret_cast<uint4*>(p.dk)[off] = make_uint4(0, 0, 0, 0);
+            reinterpret_cast<uint4*>(p.dv)[off] = make_uint4(0, 0, 0, 0);
+        }
+        return;
+    }
 
     const uint32_t sraw = smem_u32(smem_raw);
     const uint32_t sbase = (sraw + 1023u) & ~1023u;
@@ -246,7 +259,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             for (int j = 0; j < n_iter; ++j) {
                 const int s = j & 1;
                 const int h = g * G + j / nm;
-                const int m = n + j % nm;
+                const int m = m_first + j % nm;
                 const int qtok = tok0 + m * TILE;
                 // Q(j), lse(j), D(j): stage s, free once every MMA of iteration j-2 has completed
                 if (j >= 2) mbar_wait(bar_qfree(s), ((j >> 1) + 1) & 1, abort_flag, status);
@@ -352,7 +365,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         uint8_t* stg_row = sgen + L::OFF_STG + row * 128;
         for (int j = 0; j < n_iter; ++j) {
             const int h = g * G + j / nm;
-            const int m = n + j % nm;
+            const int m = m_first + j % nm;
             mbar_wait(bar_dq, j & 1, abort_flag, status);
             tc_fence_after();
             uint32_t r[D];
@@ -396,19 +409,20 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const int col0 = half * 64;                        // this thread's 64 query columns
         const int kj = n * TILE + row;
         const int my_ev = (kj < T) ? mv.evict[tok0 + kj] : 0;          // 0: visible to nobody
+        const int my_first = (general && kj < T) ? mv.kfirst[tok0 + kj] : kj;   // first query that may see this key slot
         const bool key_tail = (n * TILE + TILE > T);
         const uint8_t* cls_col = mv.tile_class + mv.cls_off[b] + n;   // class of (m, n) at cls_col[m * nb]
         const float* sLse = reinterpret_cast<const float*>(sgen + L::OFF_LSE);
         const float* sDv = reinterpret_cast<const float*>(sgen + L::OFF_DVEC);
         uint8_t* sDS_row = sgen + L::OFF_DS + half * BOX_BYTES + row * 128;
         float pv[64];
-        int cls_next = cls_col[(size_t)n * nb];            // class of the tile of the next phase_p, fetched early
+        int cls_next = cls_col[(size_t)m_first * nb];      // class of the tile of the next phase_p, fetched early
 
         auto phase_p = [&](int j) {        // P^T(j) = exp2(S^T * c - lse), masked
             const int s = j & 1;
-            const int m = n + j % nm;
+            const int m = m_first + j % nm;
             const bool need_mask = (cls_next != KVS_CLASS_FULL) || key_tail || (m * TILE + TILE > T);
-            if (j + 1 < n_iter) cls_next = cls_col[(size_t)(n + (j + 1) % nm) * nb];
+            if (j + 1 < n_iter) cls_next = cls_col[(size_t)(m_first + (j + 1) % nm) * nb];
             mbar_wait(bar_ldfull(s), (j >> 1) & 1, abort_flag, status);
             mbar_wait(bar_s, j & 1, abort_flag, status);
             tc_fence_after();
@@ -433,7 +447,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
                 for (int e = 0; e < 64; ++e) {
                     const int qi = m * TILE + col0 + e;
-                    pv[e] = ((kj <= qi) && (qi < my_ev) && (qi < T)) ? pv[e] : 0.f;
+                    pv[e] = ((my_first <= qi) && (qi < my_ev) && (qi < T)) ? pv[e] : 0.f;
                 }
             }
             uint32_t pk[32];

@@ -25,13 +25,14 @@ struct MetaHeader {
     int32_t max_seqlen;
     int32_t nblk_total;    // sum over traces of ceil(T_b / 128), written on the device
     uint32_t ncls_total;   // sum over traces of nb^2
-    int32_t pad;
+    int32_t general;       // 1: every key slot carries its own first visible query (kvs_mask_meta_keys); 0: slot j is key j
 };
 
 // Byte offsets of the arrays inside meta_buf; a pure function of the three sizes so that
 // every entry point can recompute it.
 struct MetaLayout {
-    size_t blk_off, cls_off, seq_start, blk_trace, kmin, kmax, col_last, row_cnt, fwd_order, bwd_order, evict, tile_class, row_list, total;
+    size_t blk_off, cls_off, seq_start, blk_trace, kmin, kmax, fmin, fmax, col_first, col_last, row_cnt, fwd_order, bwd_order, evict, kfirst,
+        tile_class, row_list, total;
     int nb_cap;            // capacity in blocks
     size_t cls_cap;        // capacity in tiles
 };
@@ -58,11 +59,15 @@ __host__ __device__ inline MetaLayout meta_layout(int batch, int total_tokens, i
     L.blk_trace = o; o = align_up(o + sizeof(int32_t) * nb_cap, 256);
     L.kmin = o;      o = align_up(o + sizeof(int32_t) * nb_cap, 256);
     L.kmax = o;      o = align_up(o + sizeof(int32_t) * nb_cap, 256);
+    L.fmin = o;      o = align_up(o + sizeof(int32_t) * nb_cap, 256);
+    L.fmax = o;      o = align_up(o + sizeof(int32_t) * nb_cap, 256);
+    L.col_first = o; o = align_up(o + sizeof(int32_t) * nb_cap, 256);
     L.col_last = o;  o = align_up(o + sizeof(int32_t) * nb_cap, 256);
     L.row_cnt = o;   o = align_up(o + sizeof(int32_t) * nb_cap, 256);
     L.fwd_order = o; o = align_up(o + sizeof(int32_t) * nb_cap, 256);
     L.bwd_order = o; o = align_up(o + sizeof(int32_t) * nb_cap, 256);
     L.evict = o;     o = align_up(o + sizeof(int32_t) * (size_t)(total_tokens > 0 ? total_tokens : 1), 256);
+    L.kfirst = o;    o = align_up(o + sizeof(int32_t) * (size_t)(total_tokens > 0 ? total_tokens : 1), 256);
     L.tile_class = o; o = align_up(o + L.cls_cap, 256);
     L.row_list = o;  o = align_up(o + sizeof(uint16_t) * L.cls_cap, 256);
     L.total = o;
@@ -76,13 +81,17 @@ struct MetaView {
     const uint32_t* cls_off;    // [batch+1] first tile of each trace's class matrix
     const int32_t* seq_start;   // [batch+1] copy of cu_seqlens
     const int32_t* blk_trace;   // [nblk] trace of a global block
-    const int32_t* kmin;        // [nblk]
+    const int32_t* kmin;        // [nblk] min / max over the block's key slots of the eviction step
     const int32_t* kmax;        // [nblk]
-    const int32_t* col_last;    // [nblk] last query block (trace local) that sees the key block
+    const int32_t* fmin;        // [nblk] min / max over the block's key slots of the first query that may see the slot
+    const int32_t* fmax;        // [nblk]
+    const int32_t* col_first;   // [nblk] first query block (trace local) that can see the key block
+    const int32_t* col_last;    // [nblk] last query block (trace local) that sees the key block (< col_first: none does)
     const int32_t* row_cnt;     // [nblk] non-empty key blocks of a query block row
     const int32_t* fwd_order;   // [nblk] query blocks, heaviest first
     const int32_t* bwd_order;   // [nblk] key blocks, longest query range first
-    const int32_t* evict;       // [total_tokens] copy of evict_at
+    const int32_t* evict;       // [total_tokens] eviction step of every key slot (copy of evict_at / key_evict)
+    const int32_t* kfirst;      // [total_tokens] first query that may see the slot (general metadata only)
     const uint8_t* tile_class;  // [ncls]
     const uint16_t* row_list;   // [ncls] row m of trace b at cls_off[b] + m * nb
 };
@@ -97,11 +106,15 @@ inline MetaView meta_view(const void* buf, const MetaLayout& L) {
     v.blk_trace = (const int32_t*)(p + L.blk_trace);
     v.kmin = (const int32_t*)(p + L.kmin);
     v.kmax = (const int32_t*)(p + L.kmax);
+    v.fmin = (const int32_t*)(p + L.fmin);
+    v.fmax = (const int32_t*)(p + L.fmax);
+    v.col_first = (const int32_t*)(p + L.col_first);
     v.col_last = (const int32_t*)(p + L.col_last);
     v.row_cnt = (const int32_t*)(p + L.row_cnt);
     v.fwd_order = (const int32_t*)(p + L.fwd_order);
     v.bwd_order = (const int32_t*)(p + L.bwd_order);
     v.evict = (const int32_t*)(p + L.evict);
+    v.kfirst = (const int32_t*)(p + L.kfirst);
     v.tile_class = (const uint8_t*)(p + L.tile_class);
     v.row_list = (const uint16_t*)(p + L.row_list);
     return v;

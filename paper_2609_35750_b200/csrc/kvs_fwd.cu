@@ -34,8 +34,9 @@ struct FwdSmem {
     static constexpr int TB = TILE * D * 2;
     static constexpr int OFF_Q = 0;                      // 2 query tiles
     static constexpr int OFF_KV = 2 * TB;                // 2 stages x (K, V)
-    static constexpr int OFF_EV = OFF_KV + 4 * TB;       // 2 stages x 128 int32
-    static constexpr int OFF_FLAG = OFF_EV + 2 * TILE * 4;   // 2 stages x need_mask
+    static constexpr int OFF_EV = OFF_KV + 4 * TB;       // 2 stages x 128 int32: eviction step of the stage's key slots
+    static constexpr int OFF_KF = OFF_EV + 2 * TILE * 4; // 2 stages x 128 int32: first query that may see the slot
+    static constexpr int OFF_FLAG = OFF_KF + 2 * TILE * 4;   // 2 stages x need_mask
     static constexpr int OFF_BAR = OFF_FLAG + 16;
     static constexpr int OFF_MISC = OFF_BAR + 24 * 8;
     static constexpr int TOTAL = OFF_MISC + 16;
@@ -97,6 +98,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     uint8_t* sgen = smem_raw + (sbase - sraw);
     const uint32_t sQ = sbase + L::OFF_Q, sKV = sbase + L::OFF_KV;
     int32_t* sEv = reinterpret_cast<int32_t*>(sgen + L::OFF_EV);
+    int32_t* sKf = reinterpret_cast<int32_t*>(sgen + L::OFF_KF);
+    const bool general = mv.hdr->general != 0;       // key slots carry their own first visible query (re-ordered keys)
     volatile int32_t* sFlag = reinterpret_cast<volatile int32_t*>(sgen + L::OFF_FLAG);
     uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(sgen + L::OFF_MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + L::OFF_MISC + 4);
@@ -179,6 +182,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     for (int u = 0; u < 4; ++u) {
                         const int j = n * TILE + lane * 4 + u;
                         sEv[s * TILE + lane * 4 + u] = (j < T) ? mv.evict[tok0 + j] : 0;   // 0: visible to nobody
+                        sKf[s * TILE + lane * 4 + u] = (general && j < T) ? mv.kfirst[tok0 + j] : j;
                     }
                 }
                 if (lane == 0) sFlag[s] = need_mask ? 1 : 0;
@@ -319,14 +323,27 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 
                 if (need_mask) {
                     const int4* ev4 = reinterpret_cast<const int4*>(sEv + s * TILE);
+                    if (!general) {
 #pragma unroll
-                    for (int e4 = 0; e4 < TILE / 4; ++e4) {
-                        const int4 ev = ev4[e4];
-                        const int j = n * TILE + e4 * 4;
-                        sv[e4 * 4 + 0] = ((j + 0 <= qi) && (qi < ev.x)) ? sv[e4 * 4 + 0] : -INFINITY;
-                        sv[e4 * 4 + 1] = ((j + 1 <= qi) && (qi < ev.y)) ? sv[e4 * 4 + 1] : -INFINITY;
-                        sv[e4 * 4 + 2] = ((j + 2 <= qi) && (qi < ev.z)) ? sv[e4 * 4 + 2] : -INFINITY;
-                        sv[e4 * 4 + 3] = ((j + 3 <= qi) && (qi < ev.w)) ? sv[e4 * 4 + 3] : -INFINITY;
+                        for (int e4 = 0; e4 < TILE / 4; ++e4) {
+                            const int4 ev = ev4[e4];
+                            const int j = n * TILE + e4 * 4;
+                            sv[e4 * 4 + 0] = ((j + 0 <= qi) && (qi < ev.x)) ? sv[e4 * 4 + 0] : -INFINITY;
+                            sv[e4 * 4 + 1] = ((j + 1 <= qi) && (qi < ev.y)) ? sv[e4 * 4 + 1] : -INFINITY;
+                            sv[e4 * 4 + 2] = ((j + 2 <= qi) && (qi < ev.z)) ? sv[e4 * 4 + 2] : -INFINITY;
+                            sv[e4 * 4 + 3] = ((j + 3 <= qi) && (qi < ev.w)) ? sv[e4 * 4 + 3] : -INFINITY;
+                        }
+                    } else {
+                        const int4* kf4 = reinterpret_cast<const int4*>(sKf + s * TILE);
+#pragma unroll
+                        for (int e4 = 0; e4 < TILE / 4; ++e4) {
+                            const int4 ev = ev4[e4];
+                            const int4 kf = kf4[e4];
+                            sv[e4 * 4 + 0] = ((kf.x <= qi) && (qi < ev.x)) ? sv[e4 * 4 + 0] : -INFINITY;
+                            sv[e4 * 4 + 1] = ((kf.y <= qi) && (qi < ev.y)) ? sv[e4 * 4 + 1] : -INFINITY;
+                            sv[e4 * 4 + 2] = ((kf.z <= qi) && (qi < ev.z)) ? sv[e4 * 4 + 2] : -INFINITY;
+                            sv[e4 * 4 + 3] = ((kf.w <= qi) && (qi < ev.w)) ? sv[e4 * 4 + 3] : -INFINITY;
+                        }
                     }
                 }
                 __syncwarp();

@@ -9,7 +9,8 @@
 // cost it nothing.  384 threads:
 //   warps 0-3   softmax, keys  0..63 of a block (one query row per thread)   } the two groups of a row
 //   warps 4-7   softmax, keys 64..127                                        } exchange their partial maxima
-//   warp 8      producer (TMA: Q once, K and V rings of two stages; evict_at of a block by plain loads)
+//   warp 8      producer (TMA: Q once, a K ring of three stages running two key blocks ahead of a V ring of two;
+//               evict_at of a block by plain loads)
 //   warp 9      MMA issuer (all lanes walk the loop, an elected lane issues);  warps 10-11 idle
 // Tensor memory: S_a [0,128)  S_b [128,256)  O_teacher [256,256+D)  O_student [384,384+D).  The two S
 // buffers alternate, so S of block i+1 is ready when the softmax of block i ends.  The probabilities
@@ -30,13 +31,13 @@ template <int D>
 struct DualSmem {
     static constexpr int TB = TILE * D * 2;
     static constexpr int OFF_Q = 0;
-    static constexpr int OFF_K = TB;                       // 2 stages
-    static constexpr int OFF_V = 3 * TB;                   // 2 stages
-    static constexpr int OFF_EV = 5 * TB;                  // 2 stages x 128 int32
+    static constexpr int OFF_K = TB;                       // 3 stages
+    static constexpr int OFF_V = 4 * TB;                   // 2 stages
+    static constexpr int OFF_EV = 6 * TB;                  // 2 stages x 128 int32
     static constexpr int OFF_MAX = OFF_EV + 2 * TILE * 4;  // [2 buffers][teacher, student][2 groups][128 rows] fp32
     static constexpr int OFF_FLAG = OFF_MAX + 2 * 2 * 2 * TILE * 4;
     static constexpr int OFF_BAR = OFF_FLAG + 16;
-    static constexpr int OFF_MISC = OFF_BAR + 24 * 8;
+    static constexpr int OFF_MISC = OFF_BAR + 24 * 8;      // 21 barriers in use
     static constexpr int TOTAL = OFF_MISC + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;         // slack for the 1024-byte alignment
 };
@@ -76,6 +77,10 @@ fwd_dual_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) set_status(&mv.hdr->status, KVS_ERR_BAD_META);
         return;
     }
+    if (mv.hdr->general) {          // the teacher's mask is defined for keys in their original order only
+        if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) set_status(&mv.hdr->status, KVS_ERR_UNSUPPORTED);
+        return;
+    }
     const int nblk = mv.hdr->nblk_total;
     if ((int)blockIdx.x >= nblk) return;
     const int gb = nblk - 1 - (int)blockIdx.x;       // late query blocks (the long walks) first
@@ -101,24 +106,26 @@ fwd_dual_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + L::OFF_MISC + 4);
     const uint32_t bars = sbase + L::OFF_BAR;
     const uint32_t bar_q = bars;
-    auto bar_kfull = [&](int s) { return bars + 8 * (1 + s); };
-    auto bar_vfull = [&](int s) { return bars + 8 * (3 + s); };
-    auto bar_kfree = [&](int s) { return bars + 8 * (5 + s); };     // the Q K^T product reading the stage's K has completed
-    auto bar_vfree = [&](int s) { return bars + 8 * (7 + s); };     // the P V products reading the stage's V have completed
-    auto bar_evfull = [&](int s) { return bars + 8 * (9 + s); };    // flags + evict_at of the stage (32 arrivals)
-    auto bar_evfree = [&](int s) { return bars + 8 * (11 + s); };   // the softmax warps are done with them (8 arrivals)
-    auto bar_s = [&](int t) { return bars + 8 * (13 + t); };        // S buffer t holds a fresh Q K^T
-    auto bar_p = [&](int t) { return bars + 8 * (15 + t); };        // probabilities written over S buffer t (8 arrivals)
-    const uint32_t bar_o = bars + 8 * 17;                            // every P V product issued so far has completed
-    const uint32_t bar_done = bars + 8 * 18;
+    auto bar_vfull = [&](int s) { return bars + 8 * (1 + s); };
+    auto bar_vfree = [&](int s) { return bars + 8 * (3 + s); };     // the P V products reading the stage's V have completed
+    auto bar_evfull = [&](int s) { return bars + 8 * (5 + s); };    // flags + evict_at of the stage (32 arrivals)
+    auto bar_evfree = [&](int s) { return bars + 8 * (7 + s); };    // the softmax warps are done with them (8 arrivals)
+    auto bar_s = [&](int t) { return bars + 8 * (9 + t); };         // S buffer t holds a fresh Q K^T
+    auto bar_p = [&](int t) { return bars + 8 * (11 + t); };        // probabilities written over S buffer t (8 arrivals)
+    const uint32_t bar_o = bars + 8 * 13;                            // every P V product issued so far has completed
+    const uint32_t bar_done = bars + 8 * 14;
+    auto bar_kfull = [&](int s) { return bars + 8 * (15 + s); };    // K ring of three stages: key block i sits in stage i % 3
+    auto bar_kfree = [&](int s) { return bars + 8 * (18 + s); };    // the Q K^T product reading the stage's K has completed
 
     if (tid == 0) {
         *abort_flag = 0;
         mbar_init(bar_q, 1);
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < 3; ++s) {
             mbar_init(bar_kfull(s), 1);
-            mbar_init(bar_vfull(s), 1);
             mbar_init(bar_kfree(s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar_vfull(s), 1);
             mbar_init(bar_vfree(s), 1);
             mbar_init(bar_evfull(s), 32);
             mbar_init(bar_evfree(s), 8);
@@ -147,28 +154,30 @@ fwd_dual_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 mbar_expect_tx(bar_q, L::TB);
                 for (int c = 0; c < NBOX; ++c) tma_load_3d(sQ + c * BOX_BYTES, &tm_q, c * 64, h, tok0 + m * TILE, bar_q);
             }
+            // K runs two key blocks ahead of V (three stages): S of block i + 2 is issued as soon as the softmax of
+            // block i has ended, and a tile takes about a microsecond to arrive
             auto load_k = [&](int i) {
-                const int s = i & 1;
-                if (i >= 2) mbar_wait(bar_kfree(s), ((i >> 1) + 1) & 1, abort_flag, status);
+                const int s = i % 3;
+                if (i >= 3) mbar_wait(bar_kfree(s), (uint32_t)(i / 3 + 1) & 1, abort_flag, status);
                 if (lane == 0) {
                     mbar_expect_tx(bar_kfull(s), L::TB);
                     for (int c = 0; c < NBOX; ++c) tma_load_3d(sK + s * L::TB + c * BOX_BYTES, &tm_k, c * 64, g, tok0 + i * TILE, bar_kfull(s));
                 }
             };
-            load_k(0);
-            if (nt > 1) load_k(1);
+            for (int i = 0; i < 3 && i < nt; ++i) load_k(i);
+            int c_next = cls[0];
             for (int i = 0; i < nt; ++i) {
                 const int s = i & 1;
+                const int c = c_next;
+                if (i + 1 < nt) c_next = cls[i + 1];                 // fetched a block ahead of its use
                 if (i >= 2) {
                     mbar_wait(bar_vfree(s), ((i >> 1) + 1) & 1, abort_flag, status);
                     mbar_wait(bar_evfree(s), ((i >> 1) + 1) & 1, abort_flag, status);
                 }
                 if (lane == 0) {
                     mbar_expect_tx(bar_vfull(s), L::TB);
-                    for (int c = 0; c < NBOX; ++c) tma_load_3d(sV + s * L::TB + c * BOX_BYTES, &tm_v, c * 64, g, tok0 + i * TILE, bar_vfull(s));
+                    for (int c2 = 0; c2 < NBOX; ++c2) tma_load_3d(sV + s * L::TB + c2 * BOX_BYTES, &tm_v, c2 * 64, g, tok0 + i * TILE, bar_vfull(s));
                 }
-                if (i >= 1 && i + 1 < nt) load_k(i + 1);
-                const int c = cls[i];
                 const bool ragged = (i * TILE + TILE > T);
                 const bool mask_s = (c != KVS_CLASS_EMPTY) && ((c != KVS_CLASS_FULL) || ragged);
                 if (mask_s) {
@@ -181,6 +190,7 @@ fwd_dual_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (lane == 0)
                     sFlag[s] = (c != KVS_CLASS_EMPTY ? DF_STUDENT : 0) | (mask_s ? DF_MASK_S : 0) | ((i == m || ragged) ? DF_MASK_T : 0);
                 mbar_arrive(bar_evfull(s));
+                if (i >= 1 && i + 2 < nt) load_k(i + 2);
             }
         } else if (warp == 9) {
             // ================= MMA issuer =================
@@ -189,23 +199,22 @@ fwd_dual_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const uint64_t dK0 = smem_desc(sK, 16, 1024);
             const uint64_t dV0 = smem_desc(sV, BOX_BYTES, 1024);
             constexpr uint64_t TBU = (uint64_t)(L::TB >> 4);
-            auto issue_s = [&](int t) {               // S buffer t = Q K(stage t)^T
+            auto issue_s = [&](int i) {               // S buffer i % 2 = Q K(block i, ring stage i % 3)^T
+                const int t = i & 1, ks = i % 3;
+                mbar_wait(bar_kfull(ks), (uint32_t)(i / 3) & 1, abort_flag, status);
+                tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint64_t off = (uint64_t)(((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4);
-                    if (leader) mma_ss(tmem + t * 128, dQ0 + off, dK0 + t * TBU + off, IDESC_S, kk > 0);
+                    if (leader) mma_ss(tmem + t * 128, dQ0 + off, dK0 + ks * TBU + off, IDESC_S, kk > 0);
                 }
                 if (leader) {
                     mma_commit(bar_s(t));
-                    mma_commit(bar_kfree(t));
+                    mma_commit(bar_kfree(ks));
                 }
             };
             mbar_wait(bar_q, 0, abort_flag, status);
-            for (int t = 0; t < 2 && t < nt; ++t) {
-                mbar_wait(bar_kfull(t), 0, abort_flag, status);
-                tc_fence_after();
-                issue_s(t);
-            }
+            for (int i = 0; i < 2 && i < nt; ++i) issue_s(i);
             bool student_started = false;
             int c_next = cls[0];
             for (int i = 0; i < nt; ++i) {
@@ -231,11 +240,7 @@ fwd_dual_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     mma_commit(bar_vfree(t));
                     mma_commit(bar_o);
                 }
-                if (i + 2 < nt) {
-                    mbar_wait(bar_kfull(t), (uint32_t)((i + 2) >> 1) & 1, abort_flag, status);
-                    tc_fence_after();
-                    issue_s(t);
-                }
+                if (i + 2 < nt) issue_s(i + 2);
             }
             if (leader) mma_commit(bar_done);
         }
@@ -367,13 +372,14 @@ fwd_dual_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const float neg_ref_t = (ref_t == -INFINITY) ? 0.f : -ref_t;
             const float neg_ref_s = (ref_s == -INFINITY) ? 0.f : -ref_s;
             const float gap = (ref_t == -INFINITY || ref_s == -INFINITY) ? 0.f : ref_t - ref_s;
-            const bool direct = gap > DUAL_DIRECT_GAP;
-            const float cmul = direct ? 0.f : fast_exp2(gap);
+            // a whole warp takes the direct formula as soon as one of its rows needs it (it is the exact one), so
+            // the branch is uniform and the warp-wide tensor-memory stores may sit inside it
+            const bool direct = student && __any_sync(0xffffffffu, gap > DUAL_DIRECT_GAP);
             const float2 c2 = make_float2(p.scale_log2, p.scale_log2);
             const float2 nr2 = make_float2(neg_ref_t, neg_ref_t);
             uint32_t pk[32];
             float2 acc[2];
-            if (student && direct) {
+            if (direct) {
                 // rare: the references are so far apart that the teacher's values may have underflowed
                 acc[0] = acc[1] = make_float2(0.f, 0.f);
 #pragma unroll
@@ -388,22 +394,26 @@ fwd_dual_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 sum_s += s01.x + s01.y;
                 tmem_st32(tmem_S + 64 + grp * 32, pk);
             }
-            // the teacher's probabilities take the place of the logits
-#pragma unroll
-            for (int e = 0; e < 64; e += 2) {
-                const float2 x = __ffma2_rn(make_float2(sv[e], sv[e + 1]), c2, nr2);
-                sv[e] = fast_exp2(x.x);
-                sv[e + 1] = fast_exp2(x.y);
-            }
-            if (vis_t != ~0ull) {
-#pragma unroll
-                for (int e = 0; e < 64; ++e) sv[e] = ((vis_t >> e) & 1) ? sv[e] : 0.f;
-            }
+            // the teacher's probabilities take the place of the logits; summed and packed as they are formed
             acc[0] = acc[1] = make_float2(0.f, 0.f);
+            if (vis_t == ~0ull) {
 #pragma unroll
-            for (int e = 0; e < 64; e += 2) {
-                acc[(e >> 1) & 1] = __fadd2_rn(acc[(e >> 1) & 1], make_float2(sv[e], sv[e + 1]));
-                pk[e >> 1] = pack_bf16(sv[e], sv[e + 1]);
+                for (int e = 0; e < 64; e += 2) {
+                    const float2 x = __ffma2_rn(make_float2(sv[e], sv[e + 1]), c2, nr2);
+                    sv[e] = fast_exp2(x.x);
+                    sv[e + 1] = fast_exp2(x.y);
+                    acc[(e >> 1) & 1] = __fadd2_rn(acc[(e >> 1) & 1], make_float2(sv[e], sv[e + 1]));
+                    pk[e >> 1] = pack_bf16(sv[e], sv[e + 1]);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 64; e += 2) {
+                    const float2 x = __ffma2_rn(make_float2(sv[e], sv[e + 1]), c2, nr2);
+                    sv[e] = ((vis_t >> e) & 1) ? fast_exp2(x.x) : 0.f;
+                    sv[e + 1] = ((vis_t >> (e + 1)) & 1) ? fast_exp2(x.y) : 0.f;
+                    acc[(e >> 1) & 1] = __fadd2_rn(acc[(e >> 1) & 1], make_float2(sv[e], sv[e + 1]));
+                    pk[e >> 1] = pack_bf16(sv[e], sv[e + 1]);
+                }
             }
             {
                 const float2 t01 = __fadd2_rn(acc[0], acc[1]);
@@ -416,6 +426,7 @@ fwd_dual_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                     for (int e = 0; e < 64; ++e) sv[e] = ((vis_s >> e) & 1) ? sv[e] : 0.f;
                 }
+                const float cmul = fast_exp2(gap);
                 const float2 cm2 = make_float2(cmul, cmul);
                 acc[0] = acc[1] = make_float2(0.f, 0.f);
 #pragma unroll

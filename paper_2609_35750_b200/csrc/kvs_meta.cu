@@ -5,7 +5,7 @@
 namespace kvs {
 
 // ---- kernel 0: header, per-trace offsets, block -> trace table -----------------------------
-__global__ void meta_prefix_kernel(const int32_t* __restrict__ cu_seqlens, int batch, int total_tokens, int max_seqlen,
+__global__ void meta_prefix_kernel(const int32_t* __restrict__ cu_seqlens, int batch, int total_tokens, int max_seqlen, int general,
                                    MetaHeader* hdr, int32_t* blk_off, uint32_t* cls_off, int32_t* seq_start,
                                    int32_t* blk_trace, int nb_cap, unsigned long long cls_cap) {
     __shared__ int s_bad;
@@ -37,7 +37,7 @@ __global__ void meta_prefix_kernel(const int32_t* __restrict__ cu_seqlens, int b
         hdr->max_seqlen = max_seqlen;
         hdr->nblk_total = (int32_t)nblk;
         hdr->ncls_total = (uint32_t)ncls;
-        hdr->pad = 0;
+        hdr->general = general;
         s_bad = bad;
     }
     __syncthreads();
@@ -48,10 +48,14 @@ __global__ void meta_prefix_kernel(const int32_t* __restrict__ cu_seqlens, int b
     }
 }
 
-// ---- kernel 1: one warp per key block: min / max of evict_at, validity ---------------------
-__global__ void meta_minmax_kernel(const int32_t* __restrict__ evict_at, MetaHeader* hdr, const int32_t* __restrict__ blk_off,
-                                   const int32_t* __restrict__ seq_start, const int32_t* __restrict__ blk_trace,
-                                   int32_t* kmin, int32_t* kmax, int32_t* col_last, int32_t* evict_copy) {
+// ---- kernel 1: one warp per key block: min / max over its key slots, validity ---------------
+// Slot j of a trace holds a key that query i may read iff first[j] <= i < evict[j].  Plain metadata
+// (key_first == nullptr): first[j] = j and evict[j] > j is required.  General metadata: both arrays come
+// from the caller (keys re-ordered, or another visibility rule) and a slot may be visible to nobody.
+__global__ void meta_minmax_kernel(const int32_t* __restrict__ evict_at, const int32_t* __restrict__ key_first, MetaHeader* hdr,
+                                   const int32_t* __restrict__ blk_off, const int32_t* __restrict__ seq_start,
+                                   const int32_t* __restrict__ blk_trace, int32_t* kmin, int32_t* kmax, int32_t* fmin, int32_t* fmax,
+                                   int32_t* col_first, int32_t* col_last, int32_t* evict_copy, int32_t* first_copy) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (warp >= hdr->nblk_total) return;
@@ -60,30 +64,41 @@ __global__ void meta_minmax_kernel(const int32_t* __restrict__ evict_at, MetaHea
     const int tok0 = seq_start[b];
     const int T = seq_start[b + 1] - tok0;
     const int nb = (T + TILE - 1) / TILE;
-    int mn = INT32_MAX, mx = INT32_MIN;
+    int mn = INT32_MAX, mx = INT32_MIN, fmn = INT32_MAX, fmx = INT32_MIN;
     bool bad = false;
 #pragma unroll
     for (int t = 0; t < TILE / 32; ++t) {
         const int j = n * TILE + t * 32 + lane;
         if (j < T) {
             const int e = evict_at[tok0 + j];
+            const int f = key_first ? key_first[tok0 + j] : j;
             evict_copy[tok0 + j] = e;
-            bad |= (e <= j);
+            if (key_first) first_copy[tok0 + j] = f;
+            bad |= key_first ? (f < 0) : (e <= j);
             mn = min(mn, e);
             mx = max(mx, e);
+            fmn = min(fmn, f);
+            fmx = max(fmx, f);
         }
     }
     mn = __reduce_min_sync(0xffffffffu, mn);
     mx = __reduce_max_sync(0xffffffffu, mx);
+    fmn = __reduce_min_sync(0xffffffffu, fmn);
+    fmx = __reduce_max_sync(0xffffffffu, fmx);
     const unsigned any_bad = __ballot_sync(0xffffffffu, bad);
     if (lane == 0) {
         kmin[warp] = mn;
         kmax[warp] = mx;
-        // last query block whose first row q0 = 128 m is still below kmax
+        fmin[warp] = fmn;
+        fmax[warp] = fmx;
+        // last query block whose first row q0 = 128 m is still below kmax; first one whose last row reaches fmin
         long long last = ((long long)mx - 1) / TILE;
         if (last > nb - 1) last = nb - 1;
-        if (last < n) last = n;
-        col_last[warp] = (int32_t)last;
+        long long first = fmn / TILE;
+        if (first > nb) first = nb;
+        if (!key_first && last < n) last = n;
+        col_first[warp] = (int32_t)first;
+        col_last[warp] = (mx <= 0) ? -1 : (int32_t)last;
         if (any_bad) set_status(&hdr->status, KVS_ERR_BAD_EVICT);
     }
 }
@@ -92,6 +107,7 @@ __global__ void meta_minmax_kernel(const int32_t* __restrict__ evict_at, MetaHea
 __global__ void meta_classify_kernel(MetaHeader* hdr, const int32_t* __restrict__ blk_off, const uint32_t* __restrict__ cls_off,
                                      const int32_t* __restrict__ seq_start, const int32_t* __restrict__ blk_trace,
                                      const int32_t* __restrict__ kmin, const int32_t* __restrict__ kmax,
+                                     const int32_t* __restrict__ fmin, const int32_t* __restrict__ fmax,
                                      uint8_t* tile_class, uint16_t* row_list, int32_t* row_cnt) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
@@ -110,11 +126,12 @@ __global__ void meta_classify_kernel(MetaHeader* hdr, const int32_t* __restrict_
         const int n = n0 + lane;
         int c = KVS_CLASS_EMPTY;
         if (n < nb) {
-            const int k0 = n * TILE;
-            const int k1 = min(k0 + TILE - 1, T - 1);
+            // f0, f1: the earliest / latest "first query that may see the slot" of the block; for plain
+            // metadata these are the block's first and last valid key, k0 and k1
+            const int f0 = fmin[base + n], f1 = fmax[base + n];
             const int mn = kmin[base + n], mx = kmax[base + n];
-            if (k0 > q1 || q0 >= mx) c = KVS_CLASS_EMPTY;
-            else if (k1 <= q0 && q1 < mn) c = KVS_CLASS_FULL;
+            if (f0 > q1 || q0 >= mx) c = KVS_CLASS_EMPTY;
+            else if (f1 <= q0 && q1 < mn) c = KVS_CLASS_FULL;
             else c = KVS_CLASS_PARTIAL;
             cls_row[n] = (uint8_t)c;
         }
@@ -131,9 +148,8 @@ __global__ void meta_classify_kernel(MetaHeader* hdr, const int32_t* __restrict_
 // Only the launch order of work depends on it; ties keep their order in the batch.
 constexpr int ORDER_BINS = 4096;
 __global__ void __launch_bounds__(1024)
-meta_order_kernel(MetaHeader* hdr, const int32_t* __restrict__ blk_off, const int32_t* __restrict__ blk_trace,
-                  const int32_t* __restrict__ row_cnt, const int32_t* __restrict__ col_last, int32_t* fwd_order,
-                  int32_t* bwd_order) {
+meta_order_kernel(MetaHeader* hdr, const int32_t* __restrict__ row_cnt, const int32_t* __restrict__ col_first,
+                  const int32_t* __restrict__ col_last, int32_t* fwd_order, int32_t* bwd_order) {
     __shared__ int bins[ORDER_BINS];
     __shared__ int warp_tot[32];
     const int n = hdr->nblk_total;
@@ -142,7 +158,7 @@ meta_order_kernel(MetaHeader* hdr, const int32_t* __restrict__ blk_off, const in
     auto key = [&](int i) {
         // coarse buckets (16 tiles): exact lengths would interleave blocks from all over the batch,
         // coarse ones keep runs of neighbouring blocks together while still starting the long ones first
-        const int k = bwd ? (col_last[i] - (i - blk_off[blk_trace[i]]) + 1) : row_cnt[i];
+        const int k = bwd ? (col_last[i] - col_first[i] + 1) : row_cnt[i];
         return min(max(k >> 4, 0), ORDER_BINS - 1);
     };
     for (int i = threadIdx.x; i < ORDER_BINS; i += blockDim.x) bins[i] = 0;
@@ -236,30 +252,129 @@ extern "C" size_t kvs_mask_meta_bytes(int batch, int total_tokens, int max_seqle
     return meta_layout(batch, total_tokens, max_seqlen).total;
 }
 
-extern "C" int kvs_mask_meta(const int32_t* evict_at, const int32_t* cu_seqlens, int batch, int total_tokens, int max_seqlen,
-                             void* meta_buf, size_t meta_bytes, kvs_stream_t stream) {
+namespace {
+int launch_mask_meta(const int32_t* key_evict, const int32_t* key_first, const int32_t* cu_seqlens, int batch, int total_tokens,
+                     int max_seqlen, void* meta_buf, size_t meta_bytes, kvs_stream_t stream) {
     if (!cu_seqlens || !meta_buf || batch < 0 || total_tokens < 0 || max_seqlen < 0) return KVS_ERR_INVALID_ARG;
-    if (total_tokens > 0 && !evict_at) return KVS_ERR_INVALID_ARG;
+    if (total_tokens > 0 && !key_evict) return KVS_ERR_INVALID_ARG;
     if (max_seqlen > total_tokens) max_seqlen = total_tokens;
     if (((uintptr_t)meta_buf & 255) != 0) return KVS_ERR_ALIGNMENT;
-    if (((uintptr_t)evict_at & 3) != 0 || ((uintptr_t)cu_seqlens & 3) != 0) return KVS_ERR_ALIGNMENT;
+    if (((uintptr_t)key_evict & 3) != 0 || ((uintptr_t)key_first & 3) != 0 || ((uintptr_t)cu_seqlens & 3) != 0) return KVS_ERR_ALIGNMENT;
     if ((long long)((max_seqlen + TILE - 1) / TILE) > 65535) return KVS_ERR_UNSUPPORTED;
     const MetaLayout L = meta_layout(batch, total_tokens, max_seqlen);
     if (L.cls_cap > 0xFFFFFFF0ull) return KVS_ERR_UNSUPPORTED;
     if (meta_bytes < L.total) return KVS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     MetaView v = meta_view(meta_buf, L);
-    meta_prefix_kernel<<<1, 256, 0, st>>>(cu_seqlens, batch, total_tokens, max_seqlen, v.hdr, (int32_t*)v.blk_off,
+    meta_prefix_kernel<<<1, 256, 0, st>>>(cu_seqlens, batch, total_tokens, max_seqlen, key_first ? 1 : 0, v.hdr, (int32_t*)v.blk_off,
                                           (uint32_t*)v.cls_off, (int32_t*)v.seq_start, (int32_t*)v.blk_trace, L.nb_cap,
                                           (unsigned long long)L.cls_cap);
     const int warps_per_cta = 8;
     const int grid = (L.nb_cap + warps_per_cta - 1) / warps_per_cta;
-    meta_minmax_kernel<<<grid, warps_per_cta * 32, 0, st>>>(evict_at, v.hdr, v.blk_off, v.seq_start, v.blk_trace, (int32_t*)v.kmin,
-                                                            (int32_t*)v.kmax, (int32_t*)v.col_last, (int32_t*)v.evict);
+    meta_minmax_kernel<<<grid, warps_per_cta * 32, 0, st>>>(key_evict, key_first, v.hdr, v.blk_off, v.seq_start, v.blk_trace,
+                                                            (int32_t*)v.kmin, (int32_t*)v.kmax, (int32_t*)v.fmin, (int32_t*)v.fmax,
+                                                            (int32_t*)v.col_first, (int32_t*)v.col_last, (int32_t*)v.evict,
+                                                            (int32_t*)v.kfirst);
     meta_classify_kernel<<<grid, warps_per_cta * 32, 0, st>>>(v.hdr, v.blk_off, v.cls_off, v.seq_start, v.blk_trace, v.kmin, v.kmax,
-                                                              (uint8_t*)v.tile_class, (uint16_t*)v.row_list, (int32_t*)v.row_cnt);
-    meta_order_kernel<<<2, 1024, 0, st>>>(v.hdr, v.blk_off, v.blk_trace, v.row_cnt, v.col_last, (int32_t*)v.fwd_order,
-                                          (int32_t*)v.bwd_order);
+                                                              v.fmin, v.fmax, (uint8_t*)v.tile_class, (uint16_t*)v.row_list,
+                                                              (int32_t*)v.row_cnt);
+    meta_order_kernel<<<2, 1024, 0, st>>>(v.hdr, v.row_cnt, v.col_first, v.col_last, (int32_t*)v.fwd_order, (int32_t*)v.bwd_order);
+    return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
+}
+}  // namespace
+
+extern "C" int kvs_mask_meta(const int32_t* evict_at, const int32_t* cu_seqlens, int batch, int total_tokens, int max_seqlen,
+                             void* meta_buf, size_t meta_bytes, kvs_stream_t stream) {
+    return launch_mask_meta(evict_at, nullptr, cu_seqlens, batch, total_tokens, max_seqlen, meta_buf, meta_bytes, stream);
+}
+
+extern "C" int kvs_mask_meta_keys(const int32_t* key_first, const int32_t* key_evict, const int32_t* cu_seqlens, int batch,
+                                  int total_tokens, int max_seqlen, void* meta_buf, size_t meta_bytes, kvs_stream_t stream) {
+    if (total_tokens > 0 && !key_first) return KVS_ERR_INVALID_ARG;
+    return launch_mask_meta(key_evict, key_first, cu_seqlens, batch, total_tokens, max_seqlen, meta_buf, meta_bytes, stream);
+}
+
+// ---- key re-ordering for token-level eviction ------------------------------------------------------
+namespace kvs {
+constexpr int REORDER_MAX_WINDOW = 4096;
+// One CTA per (window, trace): the window's keys sorted by (eviction step, index) with a bitonic network in shared memory.
+__global__ void __launch_bounds__(1024)
+reorder_sort_kernel(const int32_t* __restrict__ evict_at, const int32_t* __restrict__ cu_seqlens, int window, int32_t* perm,
+                    int32_t* key_first, int32_t* key_evict) {
+    __shared__ unsigned long long keys[REORDER_MAX_WINDOW];
+    const int b = blockIdx.y;
+    const int tok0 = cu_seqlens[b];
+    const int T = cu_seqlens[b + 1] - tok0;
+    const int w0 = blockIdx.x * window;
+    if (w0 >= T) return;
+    const int n = min(window, T - w0);
+    int cap = 1;
+    while (cap < n) cap <<= 1;
+    for (int i = threadIdx.x; i < cap; i += blockDim.x)
+        keys[i] = (i < n) ? (((unsigned long long)(uint32_t)evict_at[tok0 + w0 + i] << 32) | (uint32_t)i) : ~0ull;
+    __syncthreads();
+    for (int k = 2; k <= cap; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = threadIdx.x; i < cap; i += blockDim.x) {
+                const int l = i ^ j;
+                if (l > i) {
+                    const unsigned long long a = keys[i], c = keys[l];
+                    const bool up = (i & k) == 0;
+                    if ((a > c) == up) {
+                        keys[i] = c;
+                        keys[l] = a;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const int src = w0 + (int)(uint32_t)keys[i];           // trace-local index of the key that lands in slot w0 + i
+        perm[tok0 + w0 + i] = tok0 + src;
+        key_first[tok0 + w0 + i] = src;
+        key_evict[tok0 + w0 + i] = (int32_t)(keys[i] >> 32);
+    }
+}
+
+// dst row r = src row perm[r] (inverse == 0) or dst row perm[r] = src row r (inverse != 0); 16 bytes per lane
+__global__ void permute_rows_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ perm, uint4* __restrict__ dst,
+                                    long long n_rows, int row_vec, int inverse) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long r = idx / row_vec;
+    const int c = (int)(idx % row_vec);
+    if (r >= n_rows) return;
+    const long long p = perm[r];
+    if (inverse) dst[p * row_vec + c] = src[r * row_vec + c];
+    else dst[r * row_vec + c] = src[p * row_vec + c];
+}
+}  // namespace kvs
+
+extern "C" int kvs_reorder_keys(const int32_t* evict_at, const int32_t* cu_seqlens, int batch, int total_tokens, int max_seqlen,
+                                int window, int32_t* perm, int32_t* key_first, int32_t* key_evict, kvs_stream_t stream) {
+    if (batch < 0 || total_tokens < 0 || max_seqlen < 0) return KVS_ERR_INVALID_ARG;
+    if (window < 1 || window > REORDER_MAX_WINDOW) return KVS_ERR_UNSUPPORTED;
+    if (total_tokens == 0 || batch == 0) return KVS_OK;
+    if (!evict_at || !cu_seqlens || !perm || !key_first || !key_evict) return KVS_ERR_INVALID_ARG;
+    if (batch > 65535) return KVS_ERR_UNSUPPORTED;
+    if (max_seqlen > total_tokens) max_seqlen = total_tokens;
+    const int nwin = (max_seqlen + window - 1) / window;
+    dim3 grid(nwin > 0 ? nwin : 1, batch, 1);
+    reorder_sort_kernel<<<grid, 1024, 0, (cudaStream_t)stream>>>(evict_at, cu_seqlens, window, perm, key_first, key_evict);
+    return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
+}
+
+extern "C" int kvs_permute_rows(const void* src, const int32_t* perm, void* dst, long long n_rows, long long row_bytes, int inverse,
+                                kvs_stream_t stream) {
+    if (n_rows < 0 || row_bytes <= 0 || row_bytes % 16 != 0 || row_bytes / 16 > 0x7fffffffLL) return KVS_ERR_INVALID_ARG;
+    if (n_rows == 0) return KVS_OK;
+    if (!src || !perm || !dst || src == dst) return KVS_ERR_INVALID_ARG;
+    if ((((uintptr_t)src | (uintptr_t)dst) & 15) != 0 || ((uintptr_t)perm & 3) != 0) return KVS_ERR_ALIGNMENT;
+    const int row_vec = (int)(row_bytes / 16);
+    const long long total = n_rows * row_vec;
+    const long long blocks = (total + 255) / 256;
+    if (blocks > 0x7fffffffLL) return KVS_ERR_UNSUPPORTED;
+    permute_rows_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>((const uint4*)src, perm, (uint4*)dst, n_rows, row_vec, inverse);
     return cudaGetLastError() == cudaSuccess ? KVS_OK : KVS_ERR_CUDA;
 }
 
@@ -289,7 +404,7 @@ extern "C" int kvs_mask_meta_export(const void* meta_buf, int batch, const int32
     if (kmax_host && nblk)
         if (cudaMemcpyAsync(kmax_host, p + L.kmax, nblk * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVS_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return KVS_ERR_CUDA;
-    if (h.magic != META_MAGIC || h.batch != batch || h.total_tokens != total_tokens) return KVS_ERR_BAD_META;
+    if (h.magic != META_MAGIC || h.batch != batch || h.total_tokens != total_tokens || h.max_seqlen != max_seqlen) return KVS_ERR_BAD_META;
     if (h.status != KVS_OK) return h.status;
     if ((size_t)h.nblk_total != nblk || (size_t)h.ncls_total != ncls) return KVS_ERR_BAD_META;
     return KVS_OK;

@@ -409,8 +409,8 @@ def run_decode(args):
 
 
 def run_dual(args):
-    """--path dual: the self-distillation forward (student under the eviction mask + full-context teacher, sharing
-    every q k^T tile) against the two single-stream forwards it replaces, on the same inputs."""
+    """--path dual: the self-distillation forward (student under the eviction mask + full-context teacher; the teacher
+    costs one more pass over the evicted keys only, then a merge) against the two plain forwards it replaces."""
     import torch
     from paper_2609_35750_b200 import binding as B
     from paper_2609_35750_b200 import workloads as W
@@ -421,11 +421,12 @@ def run_dual(args):
     cu = torch.from_numpy(w.cu_seqlens).to(dev)
     meta = B.kvs_mask_meta(ev, cu, w.max_seqlen)
     meta_c = B.kvs_mask_meta(torch.full_like(ev, int(W.INF)), cu, w.max_seqlen)
+    meta_e = B.kvs_mask_meta_evicted(ev, cu, w.max_seqlen)
     o = [torch.empty_like(q) for _ in range(2)]
     l = [torch.empty((w.Hq, w.total_tokens), dtype=torch.float32, device=dev) for _ in range(2)]
 
     def dual():
-        B.kvs_attn_fwd_dual(q, k, v, meta, w.batch, w.max_seqlen, w.softmax_scale, out_student=o[0], lse_student=l[0],
+        B.kvs_attn_fwd_dual(q, k, v, meta, meta_e, w.batch, w.max_seqlen, w.softmax_scale, out_student=o[0], lse_student=l[0],
                             out_teacher=o[1], lse_teacher=l[1])
 
     def separate():
@@ -458,7 +459,7 @@ def run_dual(args):
                       "config": {"workload": w.name, "tokens": w.total_tokens, "Hq": w.Hq, "Hkv": w.Hkv, "head_dim": w.d,
                                  "student_pairs": pairs_s, "teacher_pairs": pairs_t,
                                  "flops": "4*d*Hq*(student pairs + teacher pairs): the shared q k^T is counted once per stream"},
-                      "roofline": {"kernel": "fwd_dual_kernel", "bound": "tensor", "achieved": tf, "peak": float(peaks["bf16_tflops"]),
+                      "roofline": {"kernel": "fwd_kernel x2 + dual_merge_kernel", "bound": "tensor", "achieved": tf, "peak": float(peaks["bf16_tflops"]),
                                    "unit": "TFLOP/s", "frac": tf / float(peaks["bf16_tflops"]), "traffic": None},
                       "dtype": "bf16", "data": "synthetic"}), flush=True)
 

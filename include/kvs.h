@@ -105,7 +105,6 @@ int kvs_mask_meta(const int32_t* evict_at, const int32_t* cu_seqlens,
  * A slot may be visible to no query at all (key_first >= key_evict); a query row that sees no key gets
  * out = 0 and lse = -inf.  Per block the classes use min/max of both arrays:
  *     EMPTY if min key_first > q1 or q0 >= max key_evict;  FULL if max key_first <= q0 and q1 < min key_evict.
- * kvs_attn_fwd_dual does not accept such a buffer (its status becomes KVS_ERR_UNSUPPORTED).
  */
 int kvs_mask_meta_keys(const int32_t* key_first, const int32_t* key_evict, const int32_t* cu_seqlens,
                        int batch, int total_tokens, int max_seqlen,
@@ -155,16 +154,31 @@ int kvs_attn_fwd(const void* q, const void* k, const void* v, const void* meta_b
                  void* out, float* lse, kvs_stream_t stream);
 
 /*
- * Student and teacher forward in one pass (App. D.3 "Training Objectives", self-distillation: the
- * student is conditioned under the eviction mask, the teacher is a full-context pass of the same
- * model on the same tokens).  Both use the same q, k, v:
- *     student:  kvs_attn_fwd's result (query i reads key j iff j <= i < evict_at[j])
- *     teacher:  plain causal attention over the same trace (query i reads every key j <= i)
- * Every S = q k^T tile is formed once and feeds both softmax / P V streams; a key block that is EMPTY
- * for the student costs the student nothing.  Arguments as kvs_attn_fwd, with one (out, lse) pair per
- * stream; all four are overwritten.  meta_buf is the one kvs_mask_meta built for the eviction mask.
+ * Metadata for the keys the eviction mask no longer shows: slot j is visible to query i iff
+ * key_evict[j] <= i, i.e. from its eviction step on, for good (kvs_mask_meta_keys with key_first =
+ * key_evict and key_evict = never, without the caller having to build those arrays).  key_evict is the
+ * evict_at of kvs_mask_meta, or the key_evict of re-ordered slots.  Together with the student's visible
+ * keys these are exactly the causal keys of a query: what kvs_attn_fwd_dual needs for the teacher.
  */
-int kvs_attn_fwd_dual(const void* q, const void* k, const void* v, const void* meta_buf,
+int kvs_mask_meta_evicted(const int32_t* key_evict, const int32_t* cu_seqlens,
+                          int batch, int total_tokens, int max_seqlen,
+                          void* meta_buf, size_t meta_bytes, kvs_stream_t stream);
+
+/*
+ * Student and teacher forward of the self-distillation objective (App. D.3 "Training Objectives": the
+ * student is conditioned under the eviction mask, the teacher is a full-context pass of the same model
+ * on the same tokens).  Both use the same q, k, v:
+ *     student:  kvs_attn_fwd's result under meta_student
+ *     teacher:  attention over every key the student sees or has lost to eviction: with keys in token
+ *               order that is plain causal attention over the trace
+ * The teacher is not a second full pass: the forward runs once more over the evicted keys only
+ * (meta_evicted, from kvs_mask_meta_evicted on the same evict_at / key_evict) and the two partial results
+ * are merged row by row (lse = log(e^lse_a + e^lse_b), out = e^(lse_a - lse) out_a + e^(lse_b - lse) out_b),
+ * so a (query, key) pair is scored twice only inside tiles that are PARTIAL for the student.
+ * Arguments as kvs_attn_fwd, with one (out, lse) pair per stream, all four overwritten; the two pairs
+ * must be distinct buffers.
+ */
+int kvs_attn_fwd_dual(const void* q, const void* k, const void* v, const void* meta_student, const void* meta_evicted,
                       int batch, int total_tokens, int max_seqlen,
                       int Hq, int Hkv, int head_dim, float softmax_scale,
                       void* out_student, float* lse_student, void* out_teacher, float* lse_teacher,

@@ -41,7 +41,8 @@ SIGNATURES = {
     "kvs_permute_rows": (_i, [_vp, _vp, _vp, ctypes.c_longlong, ctypes.c_longlong, _i, _vp]),
     "kvs_mask_meta_export": (_i, [_vp, _i, _vp, _i, _i, _vp, _vp, _vp, _vp]),
     "kvs_attn_fwd": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp]),
-    "kvs_attn_fwd_dual": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp]),
+    "kvs_mask_meta_evicted": (_i, [_vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "kvs_attn_fwd_dual": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp]),
     "kvs_attn_bwd_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
     "kvs_attn_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "kvs_attn_bwd_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp,
@@ -218,9 +219,22 @@ def kvs_attn_fwd(q, k, v, meta_buf, batch: int, max_seqlen: int, softmax_scale: 
     return out, lse
 
 
-def kvs_attn_fwd_dual(q, k, v, meta_buf, batch: int, max_seqlen: int, softmax_scale: float = 0.0,
+def kvs_mask_meta_evicted(key_evict: torch.Tensor, cu_seqlens: torch.Tensor, max_seqlen: int,
+                          meta_buf: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Metadata for the keys the eviction mask no longer shows (visible from their eviction step on)."""
+    batch = cu_seqlens.numel() - 1
+    total = key_evict.numel()
+    if meta_buf is None:
+        meta_buf = torch.empty(kvs_mask_meta_bytes(batch, total, max_seqlen), dtype=torch.uint8, device=key_evict.device)
+    _check(load().kvs_mask_meta_evicted(_dev(key_evict, "key_evict", torch.int32), _dev(cu_seqlens, "cu_seqlens", torch.int32),
+                                        batch, total, max_seqlen, _dev(meta_buf, "meta_buf", torch.uint8), meta_buf.numel(),
+                                        _stream(stream)), "kvs_mask_meta_evicted")
+    return meta_buf
+
+
+def kvs_attn_fwd_dual(q, k, v, meta_student, meta_evicted, batch: int, max_seqlen: int, softmax_scale: float = 0.0,
                       out_student=None, lse_student=None, out_teacher=None, lse_teacher=None, stream=None):
-    """Student (eviction mask) and teacher (full causal context) forward sharing every q k^T tile.
+    """Student (eviction mask) and teacher (every key seen or evicted: the full causal context) forward.
     Returns (out_student, lse_student, out_teacher, lse_teacher)."""
     total, Hq, d = q.shape
     Hkv = k.shape[1]
@@ -233,11 +247,11 @@ def kvs_attn_fwd_dual(q, k, v, meta_buf, batch: int, max_seqlen: int, softmax_sc
     if lse_teacher is None:
         lse_teacher = torch.empty((Hq, total), dtype=torch.float32, device=q.device)
     _check(load().kvs_attn_fwd_dual(_dev(q, "q", torch.bfloat16), _dev(k, "k", torch.bfloat16), _dev(v, "v", torch.bfloat16),
-                                    _dev(meta_buf, "meta_buf", torch.uint8), batch, total, max_seqlen, Hq, Hkv, d,
-                                    float(softmax_scale), _dev(out_student, "out_student", torch.bfloat16),
-                                    _dev(lse_student, "lse_student", torch.float32),
-                                    _dev(out_teacher, "out_teacher", torch.bfloat16),
-                                    _dev(lse_teacher, "lse_teacher", torch.float32), _stream(stream)), "kvs_attn_fwd_dual")
+                                    _dev(meta_student, "meta_student", torch.uint8), _dev(meta_evicted, "meta_evicted", torch.uint8),
+                                    batch, total, max_seqlen, Hq, Hkv, d, float(softmax_scale),
+                                    _dev(out_student, "out_student", torch.bfloat16), _dev(lse_student, "lse_student", torch.float32),
+                                    _dev(out_teacher, "out_teacher", torch.bfloat16), _dev(lse_teacher, "lse_teacher", torch.float32),
+                                    _stream(stream)), "kvs_attn_fwd_dual")
     return out_student, lse_student, out_teacher, lse_teacher
 
 

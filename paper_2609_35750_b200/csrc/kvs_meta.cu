@@ -52,7 +52,10 @@ __global__ void meta_prefix_kernel(const int32_t* __restrict__ cu_seqlens, int b
 // Slot j of a trace holds a key that query i may read iff first[j] <= i < evict[j].  Plain metadata
 // (key_first == nullptr): first[j] = j and evict[j] > j is required.  General metadata: both arrays come
 // from the caller (keys re-ordered, or another visibility rule) and a slot may be visible to nobody.
-__global__ void meta_minmax_kernel(const int32_t* __restrict__ evict_at, const int32_t* __restrict__ key_first, MetaHeader* hdr,
+// complement != 0: the slots of the EVICTED keys: slot j becomes visible at evict_at[j] and stays (first = evict_at,
+// evict = never), i.e. the causal key set minus what the eviction mask still shows.
+__global__ void meta_minmax_kernel(const int32_t* __restrict__ evict_at, const int32_t* __restrict__ key_first, int complement,
+                                   MetaHeader* hdr,
                                    const int32_t* __restrict__ blk_off, const int32_t* __restrict__ seq_start,
                                    const int32_t* __restrict__ blk_trace, int32_t* kmin, int32_t* kmax, int32_t* fmin, int32_t* fmax,
                                    int32_t* col_first, int32_t* col_last, int32_t* evict_copy, int32_t* first_copy) {
@@ -70,11 +73,12 @@ __global__ void meta_minmax_kernel(const int32_t* __restrict__ evict_at, const i
     for (int t = 0; t < TILE / 32; ++t) {
         const int j = n * TILE + t * 32 + lane;
         if (j < T) {
-            const int e = evict_at[tok0 + j];
-            const int f = key_first ? key_first[tok0 + j] : j;
+            const int e = complement ? INT32_MAX : evict_at[tok0 + j];
+            const int f = complement ? evict_at[tok0 + j] : (key_first ? key_first[tok0 + j] : j);
+            const bool general = complement || key_first;
             evict_copy[tok0 + j] = e;
-            if (key_first) first_copy[tok0 + j] = f;
-            bad |= key_first ? (f < 0) : (e <= j);
+            if (general) first_copy[tok0 + j] = f;
+            bad |= general ? (f < 0) : (e <= j);
             mn = min(mn, e);
             mx = max(mx, e);
             fmn = min(fmn, f);
@@ -96,7 +100,7 @@ __global__ void meta_minmax_kernel(const int32_t* __restrict__ evict_at, const i
         if (last > nb - 1) last = nb - 1;
         long long first = fmn / TILE;
         if (first > nb) first = nb;
-        if (!key_first && last < n) last = n;
+        if (!key_first && !complement && last < n) last = n;
         col_first[warp] = (int32_t)first;
         col_last[warp] = (mx <= 0) ? -1 : (int32_t)last;
         if (any_bad) set_status(&hdr->status, KVS_ERR_BAD_EVICT);
@@ -253,8 +257,8 @@ extern "C" size_t kvs_mask_meta_bytes(int batch, int total_tokens, int max_seqle
 }
 
 namespace {
-int launch_mask_meta(const int32_t* key_evict, const int32_t* key_first, const int32_t* cu_seqlens, int batch, int total_tokens,
-                     int max_seqlen, void* meta_buf, size_t meta_bytes, kvs_stream_t stream) {
+int launch_mask_meta(const int32_t* key_evict, const int32_t* key_first, int complement, const int32_t* cu_seqlens, int batch,
+                     int total_tokens, int max_seqlen, void* meta_buf, size_t meta_bytes, kvs_stream_t stream) {
     if (!cu_seqlens || !meta_buf || batch < 0 || total_tokens < 0 || max_seqlen < 0) return KVS_ERR_INVALID_ARG;
     if (total_tokens > 0 && !key_evict) return KVS_ERR_INVALID_ARG;
     if (max_seqlen > total_tokens) max_seqlen = total_tokens;
@@ -266,12 +270,12 @@ int launch_mask_meta(const int32_t* key_evict, const int32_t* key_first, const i
     if (meta_bytes < L.total) return KVS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     MetaView v = meta_view(meta_buf, L);
-    meta_prefix_kernel<<<1, 256, 0, st>>>(cu_seqlens, batch, total_tokens, max_seqlen, key_first ? 1 : 0, v.hdr, (int32_t*)v.blk_off,
+    meta_prefix_kernel<<<1, 256, 0, st>>>(cu_seqlens, batch, total_tokens, max_seqlen, (key_first || complement) ? 1 : 0, v.hdr, (int32_t*)v.blk_off,
                                           (uint32_t*)v.cls_off, (int32_t*)v.seq_start, (int32_t*)v.blk_trace, L.nb_cap,
                                           (unsigned long long)L.cls_cap);
     const int warps_per_cta = 8;
     const int grid = (L.nb_cap + warps_per_cta - 1) / warps_per_cta;
-    meta_minmax_kernel<<<grid, warps_per_cta * 32, 0, st>>>(key_evict, key_first, v.hdr, v.blk_off, v.seq_start, v.blk_trace,
+    meta_minmax_kernel<<<grid, warps_per_cta * 32, 0, st>>>(key_evict, key_first, complement, v.hdr, v.blk_off, v.seq_start, v.blk_trace,
                                                             (int32_t*)v.kmin, (int32_t*)v.kmax, (int32_t*)v.fmin, (int32_t*)v.fmax,
                                                             (int32_t*)v.col_first, (int32_t*)v.col_last, (int32_t*)v.evict,
                                                             (int32_t*)v.kfirst);
@@ -285,13 +289,18 @@ int launch_mask_meta(const int32_t* key_evict, const int32_t* key_first, const i
 
 extern "C" int kvs_mask_meta(const int32_t* evict_at, const int32_t* cu_seqlens, int batch, int total_tokens, int max_seqlen,
                              void* meta_buf, size_t meta_bytes, kvs_stream_t stream) {
-    return launch_mask_meta(evict_at, nullptr, cu_seqlens, batch, total_tokens, max_seqlen, meta_buf, meta_bytes, stream);
+    return launch_mask_meta(evict_at, nullptr, 0, cu_seqlens, batch, total_tokens, max_seqlen, meta_buf, meta_bytes, stream);
 }
 
 extern "C" int kvs_mask_meta_keys(const int32_t* key_first, const int32_t* key_evict, const int32_t* cu_seqlens, int batch,
                                   int total_tokens, int max_seqlen, void* meta_buf, size_t meta_bytes, kvs_stream_t stream) {
     if (total_tokens > 0 && !key_first) return KVS_ERR_INVALID_ARG;
-    return launch_mask_meta(key_evict, key_first, cu_seqlens, batch, total_tokens, max_seqlen, meta_buf, meta_bytes, stream);
+    return launch_mask_meta(key_evict, key_first, 0, cu_seqlens, batch, total_tokens, max_seqlen, meta_buf, meta_bytes, stream);
+}
+
+extern "C" int kvs_mask_meta_evicted(const int32_t* key_evict, const int32_t* cu_seqlens, int batch, int total_tokens, int max_seqlen,
+                                     void* meta_buf, size_t meta_bytes, kvs_stream_t stream) {
+    return launch_mask_meta(key_evict, nullptr, 1, cu_seqlens, batch, total_tokens, max_seqlen, meta_buf, meta_bytes, stream);
 }
 
 // ---- key re-ordering for token-level eviction ------------------------------------------------------

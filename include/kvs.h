@@ -184,6 +184,39 @@ int kvs_attn_fwd_dual(const void* q, const void* k, const void* v, const void* m
                       void* out_student, float* lse_student, void* out_teacher, float* lse_teacher,
                       kvs_stream_t stream);
 
+/*
+ * Forward and backward on a packed projection output (the layout the QKV and its gradient GEMM work
+ * on, so that no split / concatenation copy is needed around the attention):
+ *     qkv, dqkv : [total_tokens, Hq + 2 Hkv, head_dim]; heads 0..Hq-1 are q, then Hkv heads of k, then v
+ * qkv is bf16; dqkv is bf16 or fp32 (grad_dtype) and receives dq, dk, dv in the same head order.
+ * Everything else (out, lse, dout, meta_buf, workspace, errors) as in kvs_attn_fwd / kvs_attn_bwd; the
+ * workspace size is that of kvs_attn_bwd_workspace_bytes for the same dims.
+ */
+int kvs_attn_fwd_packed(const void* qkv, const void* meta_buf,
+                        int batch, int total_tokens, int max_seqlen,
+                        int Hq, int Hkv, int head_dim, float softmax_scale,
+                        void* out, float* lse, kvs_stream_t stream);
+int kvs_attn_bwd_packed(const void* dout, const void* qkv, const void* out, const float* lse, const void* meta_buf,
+                        int batch, int total_tokens, int max_seqlen,
+                        int Hq, int Hkv, int head_dim, float softmax_scale, int grad_dtype,
+                        void* dqkv, void* workspace, size_t workspace_bytes, kvs_stream_t stream);
+
+/*
+ * Rotary position embedding of q and k (and, with inverse != 0, the transposed rotation that takes
+ * gradients with respect to the rotated tensors back to the unrotated ones).  KV-streams keeps every
+ * token's position under eviction (Sec. 2: only re-prefill compaction resets positions), so on one
+ * continuous trace a token's rotation depends on its trace index alone.  Rotate-half convention:
+ *     angle(t, c) = pos_t * theta_base^(-2c / head_dim),  c < head_dim / 2
+ *     y[c] = x[c] cos - x[c + d/2] sin;   y[c + d/2] = x[c + d/2] cos + x[c] sin
+ * q [total_tokens, Hq, head_dim], k [total_tokens, Hkv, head_dim], contiguous, bf16 (elem_dtype =
+ * KVS_GRAD_BF16) or fp32 (KVS_GRAD_FP32); either may be NULL; q_out / k_out may alias q / k.
+ * positions: int32 [total_tokens], or NULL for the trace-local index (cu_seqlens, batch then required).
+ * Angles are formed in double precision, the rotation in fp32, one rounding to the output type.
+ */
+int kvs_rope_qk(const void* q, const void* k, const int32_t* positions, const int32_t* cu_seqlens,
+                int batch, int total_tokens, int Hq, int Hkv, int head_dim, float theta_base,
+                int elem_dtype, int inverse, void* q_out, void* k_out, kvs_stream_t stream);
+
 /* Bytes needed for the backward workspace (row sums, fp32 dQ accumulator, status). */
 size_t kvs_attn_bwd_workspace_bytes(int total_tokens, int Hq, int Hkv, int head_dim, int grad_dtype);
 

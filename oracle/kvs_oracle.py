@@ -628,3 +628,33 @@ def merge_partial(out_a, lse_a, out_b, lse_b):
     wb = np.exp(lb - np.where(np.isfinite(lse), lse, 0.0)) * np.isfinite(lb)
     out = wa.T[:, :, None] * np.asarray(out_a, dtype=np.float64) + wb.T[:, :, None] * np.asarray(out_b, dtype=np.float64)
     return out, lse
+
+
+# --------------------------------------------------------------------------
+# rotary position embedding on one continuous trace
+# --------------------------------------------------------------------------
+def rope_rotate(x, positions, theta_base=10000.0, inverse=False):
+    """x [T, H, d]; positions int [T].  Rotate-half convention: for c < d/2 and angle = pos * base^(-2c/d),
+    y[c] = x[c] cos - x[c + d/2] sin,  y[c + d/2] = x[c + d/2] cos + x[c] sin.
+    KV-streams never resets positions when entries are evicted (Sec. 2), so on the training trace
+    ``positions`` is simply each token's index in its trace.  ``inverse`` rotates by the opposite angle,
+    which is the transpose: the map from gradients w.r.t. y to gradients w.r.t. x."""
+    x = np.asarray(x, dtype=np.float64)
+    T, H, d = x.shape
+    half = d // 2
+    pos = np.asarray(positions, dtype=np.float64)
+    inv_freq = theta_base ** (-2.0 * np.arange(half) / d)
+    ang = pos[:, None] * inv_freq[None, :]
+    if inverse:
+        ang = -ang
+    c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    y = np.empty_like(x)
+    y[..., :half] = x[..., :half] * c - x[..., half:] * s
+    y[..., half:] = x[..., half:] * c + x[..., :half] * s
+    return y
+
+
+def trace_positions(cu_seqlens):
+    """Trace-local index of every packed token."""
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    return np.concatenate([np.arange(cu[b + 1] - cu[b]) for b in range(len(cu) - 1)] or [np.zeros(0, np.int64)])

@@ -43,6 +43,9 @@ SIGNATURES = {
     "kvs_attn_fwd": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp]),
     "kvs_mask_meta_evicted": (_i, [_vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "kvs_attn_fwd_dual": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp, _vp, _vp]),
+    "kvs_attn_fwd_packed": (_i, [_vp, _vp, _i, _i, _i, _i, _i, _i, _f, _vp, _vp, _vp]),
+    "kvs_attn_bwd_packed": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _sz, _vp]),
+    "kvs_rope_qk": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _i, _i, _vp, _vp, _vp]),
     "kvs_attn_bwd_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
     "kvs_attn_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "kvs_attn_bwd_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp,
@@ -253,6 +256,60 @@ def kvs_attn_fwd_dual(q, k, v, meta_student, meta_evicted, batch: int, max_seqle
                                     _dev(out_teacher, "out_teacher", torch.bfloat16), _dev(lse_teacher, "lse_teacher", torch.float32),
                                     _stream(stream)), "kvs_attn_fwd_dual")
     return out_student, lse_student, out_teacher, lse_teacher
+
+
+def kvs_attn_fwd_packed(qkv, meta_buf, batch: int, max_seqlen: int, Hq: int, Hkv: int, softmax_scale: float = 0.0,
+                        out=None, lse=None, stream=None):
+    """qkv bf16 [Ttot, Hq + 2 Hkv, d] (q heads, k heads, v heads).  Returns (out [Ttot,Hq,d], lse [Hq,Ttot])."""
+    total, H, d = qkv.shape
+    if H != Hq + 2 * Hkv:
+        raise ValueError("qkv must have Hq + 2 Hkv heads")
+    if out is None:
+        out = torch.empty((total, Hq, d), dtype=torch.bfloat16, device=qkv.device)
+    if lse is None:
+        lse = torch.empty((Hq, total), dtype=torch.float32, device=qkv.device)
+    _check(load().kvs_attn_fwd_packed(_dev(qkv, "qkv", torch.bfloat16), _dev(meta_buf, "meta_buf", torch.uint8), batch, total,
+                                      max_seqlen, Hq, Hkv, d, float(softmax_scale), _dev(out, "out", torch.bfloat16),
+                                      _dev(lse, "lse", torch.float32), _stream(stream)), "kvs_attn_fwd_packed")
+    return out, lse
+
+
+def kvs_attn_bwd_packed(dout, qkv, out, lse, meta_buf, batch: int, max_seqlen: int, Hq: int, Hkv: int, softmax_scale: float = 0.0,
+                        grad_dtype: int = GRAD_FP32, dqkv=None, workspace=None, stream=None):
+    """Returns dqkv [Ttot, Hq + 2 Hkv, d] (bf16 or fp32): dq, dk, dv in the head order of qkv."""
+    total, H, d = qkv.shape
+    gdt = torch.float32 if grad_dtype == GRAD_FP32 else torch.bfloat16
+    if dqkv is None:
+        dqkv = torch.empty(qkv.shape, dtype=gdt, device=qkv.device)
+    if workspace is None:
+        workspace = torch.empty(kvs_attn_bwd_workspace_bytes(total, Hq, Hkv, d, grad_dtype), dtype=torch.uint8, device=qkv.device)
+    _check(load().kvs_attn_bwd_packed(_dev(dout, "dout", torch.bfloat16), _dev(qkv, "qkv", torch.bfloat16),
+                                      _dev(out, "out", torch.bfloat16), _dev(lse, "lse", torch.float32),
+                                      _dev(meta_buf, "meta_buf", torch.uint8), batch, total, max_seqlen, Hq, Hkv, d,
+                                      float(softmax_scale), grad_dtype, _dev(dqkv, "dqkv", gdt),
+                                      _dev(workspace, "workspace", torch.uint8), workspace.numel(), _stream(stream)),
+           "kvs_attn_bwd_packed")
+    return dqkv
+
+
+def kvs_rope_qk(q, k, cu_seqlens=None, positions=None, theta_base: float = 10000.0, inverse: bool = False, q_out=None, k_out=None,
+                stream=None):
+    """Rotary embedding of q and/or k (bf16 or fp32, [Ttot, H, d]); inverse=True applies the transposed rotation (for
+    gradients).  positions int32 [Ttot] or None for the trace-local index (cu_seqlens then required).  Returns (q_out, k_out)."""
+    ref = q if q is not None else k
+    total, _, d = ref.shape
+    dt = GRAD_FP32 if ref.dtype == torch.float32 else GRAD_BF16
+    if q is not None and q_out is None:
+        q_out = torch.empty_like(q)
+    if k is not None and k_out is None:
+        k_out = torch.empty_like(k)
+    ptr = lambda t, n: _dev(t, n, ref.dtype) if t is not None else None
+    _check(load().kvs_rope_qk(ptr(q, "q"), ptr(k, "k"), _dev(positions, "positions", torch.int32) if positions is not None else None,
+                              _dev(cu_seqlens, "cu_seqlens", torch.int32) if cu_seqlens is not None else None,
+                              (cu_seqlens.numel() - 1) if cu_seqlens is not None else 0, total,
+                              q.shape[1] if q is not None else 0, k.shape[1] if k is not None else 0, d, float(theta_base), dt,
+                              1 if inverse else 0, ptr(q_out, "q_out"), ptr(k_out, "k_out"), _stream(stream)), "kvs_rope_qk")
+    return q_out, k_out
 
 
 def kvs_attn_bwd_workspace_bytes(total_tokens: int, Hq: int, Hkv: int, head_dim: int, grad_dtype: int) -> int:

@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libkvs.so")
-SOURCES = ["kvs_api.cu", "kvs_meta.cu", "kvs_fwd.cu", "kvs_fwd_dual.cu", "kvs_bwd.cu", "kvs_bwd_noalloc.cu", "kvs_decode.cu"]
+SOURCES = ["kvs_api.cu", "kvs_meta.cu", "kvs_fwd.cu", "kvs_fwd_dual.cu", "kvs_bwd.cu", "kvs_bwd_noalloc.cu", "kvs_decode.cu", "kvs_rope.cu"]
 HEADERS = [os.path.join(CSRC, "kvs_common.cuh"), os.path.join(INCLUDE, "kvs.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I" + INCLUDE, "-I" + CSRC]

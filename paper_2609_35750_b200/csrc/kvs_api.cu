@@ -25,11 +25,12 @@ static EncodeTiledFn encode_fn() {
 
 // bf16 [total_tokens, heads, head_dim] viewed as (head_dim, heads, tokens); box = 64 columns x
 // 1 head x box_rows tokens, 128-byte swizzle, out-of-range rows read as zero.
-int make_tmap_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows) {
+int make_tmap_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows, long long token_stride) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return KVS_ERR_CUDA;
+    if (token_stride <= 0) token_stride = (long long)heads * head_dim;
     cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)heads, (cuuint64_t)total_tokens};
-    cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)heads * head_dim * 2};
+    cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)token_stride * 2};
     cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
@@ -40,11 +41,13 @@ int make_tmap_thd(CUtensorMap* map, const void* base, int total_tokens, int head
 
 // fp32 [total_tokens, heads, head_dim] viewed as (head_dim, heads, tokens); box = 32 columns (128 bytes) x
 // 1 head x box_rows tokens, 128-byte swizzle.  Used as the destination of TMA reduce-adds.
-int make_tmap_f32_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows) {
+int make_tmap_f32_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows,
+                      long long token_stride) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return KVS_ERR_CUDA;
+    if (token_stride <= 0) token_stride = (long long)heads * head_dim;
     cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)heads, (cuuint64_t)total_tokens};
-    cuuint64_t strides[2] = {(cuuint64_t)head_dim * 4, (cuuint64_t)heads * head_dim * 4};
+    cuuint64_t strides[2] = {(cuuint64_t)head_dim * 4, (cuuint64_t)token_stride * 4};
     cuuint32_t box[3] = {32, 1, (cuuint32_t)box_rows};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,

@@ -33,7 +33,7 @@ constexpr int DOT_ROWS = 4;
 template <int D>
 __global__ void __launch_bounds__(256)
 bwd_dot_kernel(const __nv_bfloat16* __restrict__ dout, const __nv_bfloat16* __restrict__ out,
-               float* __restrict__ dvec, float* __restrict__ dq_acc, int total_tokens, int Hq, WsHeader* hdr) {
+               float* __restrict__ dvec, float* __restrict__ dq_acc, long long dq_ts, int total_tokens, int Hq, WsHeader* hdr) {
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         hdr->magic = WS_MAGIC;
         hdr->status = KVS_OK;
@@ -71,7 +71,7 @@ bwd_dot_kernel(const __nv_bfloat16* __restrict__ dout, const __nv_bfloat16* __re
         for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         if (row < rows) {
             if (dq_acc) {
-                float4* z = reinterpret_cast<float4*>(dq_acc + (size_t)row * D + c * 8);
+                float4* z = reinterpret_cast<float4*>(dq_acc + (size_t)(row / Hq) * dq_ts + (size_t)(row % Hq) * D + c * 8);
                 z[0] = zero;
                 z[1] = zero;
             }
@@ -81,14 +81,16 @@ bwd_dot_kernel(const __nv_bfloat16* __restrict__ dout, const __nv_bfloat16* __re
 }
 
 // ---- post-pass --------------------------------------------------------------------------------
-__global__ void bwd_cast_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, size_t n4) {
+// acc: contiguous [tokens, row_elems]; dq: rows of row_elems elements, dq_ts elements apart
+__global__ void bwd_cast_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, size_t n4, int row_elems, long long dq_ts) {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n4) return;
     const float4 x = reinterpret_cast<const float4*>(acc)[i];
     uint2 w;
     w.x = pack_bf16(x.x, x.y);
     w.y = pack_bf16(x.z, x.w);
-    reinterpret_cast<uint2*>(dq)[i] = w;
+    const size_t e = i * 4;
+    *reinterpret_cast<uint2*>(dq + (e / row_elems) * (size_t)dq_ts + e % row_elems) = w;
 }
 
 // ---- main -------------------------------------------------------------------------------------
@@ -139,6 +141,7 @@ struct BwdParams {
     const float* dvec;
     void* dk;
     void* dv;
+    long long dkv_ts;       // elements between consecutive tokens of dk and dv
     int grad_fp32;
     int32_t* status;
 };
@@ -187,7 +190,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const int rows = min(TILE, T - n * TILE);
         const size_t per_row = (size_t)D * (p.grad_fp32 ? 4 : 2) / 16;          // 16-byte words of one (token, head) row
         for (int i = tid; i < rows * (int)per_row; i += BWD_THREADS) {
-            const size_t off = ((size_t)(tok0 + n * TILE + i / (int)per_row) * p.Hkv + g) * per_row + i % (int)per_row;
+            const size_t off = (size_t)(tok0 + n * TILE + i / (int)per_row) * (size_t)(p.dkv_ts / D) * per_row + (size_t)g * per_row + i % (int)per_row;
             reinterpret_cast<uint4*>(p.dk)[off] = make_uint4(0, 0, 0, 0);
             reinterpret_cast<uint4*>(p.dv)[off] = make_uint4(0, 0, 0, 0);
         }
@@ -504,7 +507,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         mbar_wait(bar_qfree((n_iter - 1) & 1), ((n_iter - 1) >> 1) & 1, abort_flag, status);
         tc_fence_after();
         const bool kvalid = kj < T;
-        const size_t orow = ((size_t)(tok0 + kj) * p.Hkv + g) * D + half * HALF_D;
+        const size_t orow = (size_t)(tok0 + kj) * (size_t)p.dkv_ts + (size_t)g * D + half * HALF_D;
 #pragma unroll
         for (int which = 0; which < 2; ++which) {
             const uint32_t src = (which == 0 ? tmem_dK : tmem_dV) + lane_sel + half * HALF_D;
@@ -548,7 +551,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 template <int D>
 static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                       const CUtensorMap& tdq, const MetaView& mv,
-                      const BwdParams& p, const __nv_bfloat16* dout, const __nv_bfloat16* out, float* dvec, float* dq_acc,
+                      const BwdParams& p, const __nv_bfloat16* dout, const __nv_bfloat16* out, float* dvec, float* dq_acc, long long dq_ts,
                       WsHeader* hdr, int nb_cap, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1) {
     {
         const long long rows = (long long)p.total_tokens * p.Hq;
@@ -557,7 +560,7 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
         const int threads = 256;
         const long long blocks = (warps * 32 + threads - 1) / threads;
         if (blocks > 0x7fffffffLL) return KVS_ERR_UNSUPPORTED;
-        bwd_dot_kernel<D><<<(unsigned)(blocks > 0 ? blocks : 1), threads, 0, st>>>(dout, out, dvec, dq_acc, p.total_tokens, p.Hq, hdr);
+        bwd_dot_kernel<D><<<(unsigned)(blocks > 0 ? blocks : 1), threads, 0, st>>>(dout, out, dvec, dq_acc, dq_ts, p.total_tokens, p.Hq, hdr);
     }
     auto kern = bwd_kernel<D>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::DYN_BYTES) != cudaSuccess) return KVS_ERR_CUDA;
@@ -578,10 +581,12 @@ extern "C" size_t kvs_attn_bwd_workspace_bytes(int total_tokens, int Hq, int Hkv
     return bwd_ws_layout(total_tokens, Hq, head_dim, grad_dtype).total;
 }
 
-extern "C" int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, const void* v, const void* out, const float* lse,
-                               const void* meta_buf, int batch, int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim,
-                               float softmax_scale, int grad_dtype, void* dq, void* dk, void* dv, void* workspace,
-                               size_t workspace_bytes, kvs_stream_t stream, void* event_main_begin, void* event_main_end) {
+namespace {
+// in_ts: elements between consecutive tokens of q and of k, v; g_ts: of dq and of dk, dv (0: tensors of their own)
+int bwd_impl(const void* dout, const void* q, const void* k, const void* v, long long in_ts, const void* out, const float* lse,
+             const void* meta_buf, int batch, int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim,
+             float softmax_scale, int grad_dtype, void* dq, void* dk, void* dv, long long g_ts, void* workspace,
+             size_t workspace_bytes, kvs_stream_t stream, void* event_main_begin, void* event_main_end) {
     cudaEvent_t ev0 = (cudaEvent_t)event_main_begin, ev1 = (cudaEvent_t)event_main_end;
     if (batch < 0 || total_tokens < 0 || max_seqlen < 0 || Hq <= 0 || Hkv <= 0) return KVS_ERR_INVALID_ARG;
     if (head_dim != 64 && head_dim != 128) return KVS_ERR_UNSUPPORTED;
@@ -600,9 +605,9 @@ extern "C" int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, c
     const MetaLayout L = meta_layout(batch, total_tokens, max_seqlen);
     const MetaView mv = meta_view(meta_buf, L);
     CUtensorMap tq, tk, tv, tdo, tdq;
-    if ((rc = make_tmap_thd(&tq, q, total_tokens, Hq, head_dim, TILE)) != KVS_OK) return rc;
-    if ((rc = make_tmap_thd(&tk, k, total_tokens, Hkv, head_dim, TILE)) != KVS_OK) return rc;
-    if ((rc = make_tmap_thd(&tv, v, total_tokens, Hkv, head_dim, TILE)) != KVS_OK) return rc;
+    if ((rc = make_tmap_thd(&tq, q, total_tokens, Hq, head_dim, TILE, in_ts)) != KVS_OK) return rc;
+    if ((rc = make_tmap_thd(&tk, k, total_tokens, Hkv, head_dim, TILE, in_ts)) != KVS_OK) return rc;
+    if ((rc = make_tmap_thd(&tv, v, total_tokens, Hkv, head_dim, TILE, in_ts)) != KVS_OK) return rc;
     if ((rc = make_tmap_thd(&tdo, dout, total_tokens, Hq, head_dim, TILE)) != KVS_OK) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     char* ws = (char*)workspace;
@@ -617,25 +622,54 @@ extern "C" int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, c
     p.scale_log2 = p.scale * 1.4426950408889634f;
     p.lse = lse;
     p.dvec = (const float*)(ws + W.dvec);
+    // bf16 gradients: dq is accumulated in the workspace (contiguous) and cast into place afterwards;
+    // fp32 gradients: straight into dq, whatever its token stride
+    const long long dq_ts_out = g_ts > 0 ? g_ts : (long long)Hq * head_dim;
     float* dq_acc = grad_dtype == KVS_GRAD_FP32 ? (float*)dq : (float*)(ws + W.dq_acc);
-    if ((rc = make_tmap_f32_thd(&tdq, dq_acc, total_tokens, Hq, head_dim, TILE)) != KVS_OK) return rc;
+    const long long dq_ts = grad_dtype == KVS_GRAD_FP32 ? dq_ts_out : (long long)Hq * head_dim;
+    if ((rc = make_tmap_f32_thd(&tdq, dq_acc, total_tokens, Hq, head_dim, TILE, dq_ts)) != KVS_OK) return rc;
     p.dk = dk;
     p.dv = dv;
+    p.dkv_ts = g_ts > 0 ? g_ts : (long long)Hkv * head_dim;
     p.grad_fp32 = grad_dtype == KVS_GRAD_FP32;
     p.status = &((WsHeader*)ws)->status;
     rc = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, tdq, mv, p, (const __nv_bfloat16*)dout, (const __nv_bfloat16*)out, (float*)(ws + W.dvec),
-                                         dq_acc, (WsHeader*)ws, L.nb_cap, st, ev0, ev1)
+                                         dq_acc, dq_ts, (WsHeader*)ws, L.nb_cap, st, ev0, ev1)
                         : launch_bwd<128>(tq, tk, tv, tdo, tdq, mv, p, (const __nv_bfloat16*)dout, (const __nv_bfloat16*)out,
-                                          (float*)(ws + W.dvec), dq_acc, (WsHeader*)ws, L.nb_cap, st, ev0, ev1);
+                                          (float*)(ws + W.dvec), dq_acc, dq_ts, (WsHeader*)ws, L.nb_cap, st, ev0, ev1);
     if (rc != KVS_OK) return rc;
     if (grad_dtype == KVS_GRAD_BF16) {
         const size_t n4 = nq / 4;
         const size_t blocks = (n4 + 255) / 256;
         if (blocks > 0x7fffffffull) return KVS_ERR_UNSUPPORTED;
-        bwd_cast_kernel<<<(unsigned)blocks, 256, 0, st>>>(dq_acc, (__nv_bfloat16*)dq, n4);
+        bwd_cast_kernel<<<(unsigned)blocks, 256, 0, st>>>(dq_acc, (__nv_bfloat16*)dq, n4, Hq * head_dim, dq_ts_out);
         if (cudaGetLastError() != cudaSuccess) return KVS_ERR_CUDA;
     }
     return KVS_OK;
+}
+}  // namespace
+
+extern "C" int kvs_attn_bwd_ex(const void* dout, const void* q, const void* k, const void* v, const void* out, const float* lse,
+                               const void* meta_buf, int batch, int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim,
+                               float softmax_scale, int grad_dtype, void* dq, void* dk, void* dv, void* workspace,
+                               size_t workspace_bytes, kvs_stream_t stream, void* event_main_begin, void* event_main_end) {
+    return bwd_impl(dout, q, k, v, 0, out, lse, meta_buf, batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, softmax_scale, grad_dtype,
+                    dq, dk, dv, 0, workspace, workspace_bytes, stream, event_main_begin, event_main_end);
+}
+
+extern "C" int kvs_attn_bwd_packed(const void* dout, const void* qkv, const void* out, const float* lse, const void* meta_buf,
+                                   int batch, int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim, float softmax_scale,
+                                   int grad_dtype, void* dqkv, void* workspace, size_t workspace_bytes, kvs_stream_t stream) {
+    if (Hq <= 0 || Hkv <= 0 || head_dim <= 0) return KVS_ERR_INVALID_ARG;
+    if (grad_dtype != KVS_GRAD_BF16 && grad_dtype != KVS_GRAD_FP32) return KVS_ERR_INVALID_ARG;
+    if (total_tokens > 0 && batch > 0 && (!qkv || !dqkv)) return KVS_ERR_INVALID_ARG;
+    const long long ts = (long long)(Hq + 2 * Hkv) * head_dim;
+    const size_t gsz = grad_dtype == KVS_GRAD_FP32 ? 4 : 2;
+    const char* in = (const char*)qkv;
+    char* g = (char*)dqkv;
+    return bwd_impl(dout, in, in + (size_t)Hq * head_dim * 2, in + (size_t)(Hq + Hkv) * head_dim * 2, ts, out, lse, meta_buf, batch,
+                    total_tokens, max_seqlen, Hq, Hkv, head_dim, softmax_scale, grad_dtype, g, g + (size_t)Hq * head_dim * gsz,
+                    g + (size_t)(Hq + Hkv) * head_dim * gsz, ts, workspace, workspace_bytes, stream, nullptr, nullptr);
 }
 
 extern "C" int kvs_attn_bwd(const void* dout, const void* q, const void* k, const void* v, const void* out, const float* lse,

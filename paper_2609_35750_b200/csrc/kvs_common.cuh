@@ -128,8 +128,11 @@ struct WsHeader {
 };
 
 // Host helpers implemented in kvs_api.cu
-int make_tmap_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows);
-int make_tmap_f32_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows);
+// token_stride: elements between consecutive tokens (0: heads * head_dim, i.e. a tensor of its own; larger when the
+// tensor is a slice of heads of a packed [tokens, all heads, head_dim] buffer)
+int make_tmap_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows, long long token_stride = 0);
+int make_tmap_f32_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows,
+                      long long token_stride = 0);
 int check_device_sm100();
 
 #ifdef __CUDACC__

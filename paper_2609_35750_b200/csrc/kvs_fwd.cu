@@ -522,9 +522,11 @@ static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
 
 using namespace kvs;
 
-extern "C" int kvs_attn_fwd(const void* q, const void* k, const void* v, const void* meta_buf, int batch, int total_tokens,
-                            int max_seqlen, int Hq, int Hkv, int head_dim, float softmax_scale, void* out, float* lse,
-                            kvs_stream_t stream) {
+namespace {
+// q_ts / kv_ts: elements between consecutive tokens of q and of k, v (0: tensors of their own)
+int fwd_impl(const void* q, const void* k, const void* v, long long q_ts, long long kv_ts, const void* meta_buf, int batch,
+             int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim, float softmax_scale, void* out, float* lse,
+             kvs_stream_t stream) {
     if (batch < 0 || total_tokens < 0 || max_seqlen < 0 || Hq <= 0 || Hkv <= 0) return KVS_ERR_INVALID_ARG;
     if (head_dim != 64 && head_dim != 128) return KVS_ERR_UNSUPPORTED;
     if (Hq % Hkv != 0 || Hq > 65535) return KVS_ERR_UNSUPPORTED;
@@ -538,9 +540,9 @@ extern "C" int kvs_attn_fwd(const void* q, const void* k, const void* v, const v
     const MetaLayout L = meta_layout(batch, total_tokens, max_seqlen);
     const MetaView mv = meta_view(meta_buf, L);
     CUtensorMap tq, tk, tv;
-    if ((rc = make_tmap_thd(&tq, q, total_tokens, Hq, head_dim, TILE)) != KVS_OK) return rc;
-    if ((rc = make_tmap_thd(&tk, k, total_tokens, Hkv, head_dim, TILE)) != KVS_OK) return rc;
-    if ((rc = make_tmap_thd(&tv, v, total_tokens, Hkv, head_dim, TILE)) != KVS_OK) return rc;
+    if ((rc = make_tmap_thd(&tq, q, total_tokens, Hq, head_dim, TILE, q_ts)) != KVS_OK) return rc;
+    if ((rc = make_tmap_thd(&tk, k, total_tokens, Hkv, head_dim, TILE, kv_ts)) != KVS_OK) return rc;
+    if ((rc = make_tmap_thd(&tv, v, total_tokens, Hkv, head_dim, TILE, kv_ts)) != KVS_OK) return rc;
     FwdParams p;
     p.batch = batch;
     p.total_tokens = total_tokens;
@@ -554,4 +556,20 @@ extern "C" int kvs_attn_fwd(const void* q, const void* k, const void* v, const v
     cudaStream_t st = (cudaStream_t)stream;
     return head_dim == 64 ? launch_fwd<64>(tq, tk, tv, mv, p, L.nb_cap, st) : launch_fwd<128>(tq, tk, tv, mv, p, L.nb_cap, st);
 }
+}  // namespace
 
+extern "C" int kvs_attn_fwd(const void* q, const void* k, const void* v, const void* meta_buf, int batch, int total_tokens,
+                            int max_seqlen, int Hq, int Hkv, int head_dim, float softmax_scale, void* out, float* lse,
+                            kvs_stream_t stream) {
+    return fwd_impl(q, k, v, 0, 0, meta_buf, batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, softmax_scale, out, lse, stream);
+}
+
+extern "C" int kvs_attn_fwd_packed(const void* qkv, const void* meta_buf, int batch, int total_tokens, int max_seqlen, int Hq,
+                                   int Hkv, int head_dim, float softmax_scale, void* out, float* lse, kvs_stream_t stream) {
+    if (Hq <= 0 || Hkv <= 0 || head_dim <= 0) return KVS_ERR_INVALID_ARG;
+    if (total_tokens > 0 && batch > 0 && !qkv) return KVS_ERR_INVALID_ARG;
+    const long long ts = (long long)(Hq + 2 * Hkv) * head_dim;
+    const char* base = (const char*)qkv;
+    return fwd_impl(base, base + (size_t)Hq * head_dim * 2, base + (size_t)(Hq + Hkv) * head_dim * 2, ts, ts, meta_buf, batch,
+                    total_tokens, max_seqlen, Hq, Hkv, head_dim, softmax_scale, out, lse, stream);
+}

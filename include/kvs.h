@@ -96,7 +96,7 @@ int kvs_mask_meta(const int32_t* evict_at, const int32_t* cu_seqlens,
  * Mask metadata for key slots that carry their own visibility interval: slot j of a trace holds a key
  * that query i of the trace may read iff  key_first[j] <= i < key_evict[j]  (both int32 [total_tokens],
  * trace-local).  kvs_mask_meta is the case key_first[j] = j.  Two uses:
- *   - token-level eviction (App. A.4): with the keys of a trace re-ordered by kvs_reorder_keys, the
+ *   - token-level eviction (App. B.4): with the keys of a trace re-ordered by kvs_reorder_keys, the
  *     slots of a 128-slot block die at about the same time, so most tiles are FULL or EMPTY instead of
  *     PARTIAL; the attention calls then take k, v in the re-ordered slot order (kvs_permute_rows) and
  *     return dk, dv in that order;
@@ -111,7 +111,7 @@ int kvs_mask_meta_keys(const int32_t* key_first, const int32_t* key_evict, const
                        void* meta_buf, size_t meta_bytes, kvs_stream_t stream);
 
 /*
- * Key order for token-level eviction (App. A.4 "Turn-Wise Compaction" discusses token-level eviction):
+ * Key order for token-level eviction (App. B.4 "Turn-Wise Compaction" discusses token-level eviction):
  * attention does not depend on the order of its keys, so the keys of a trace may be stored in any order
  * as long as each carries its index and its eviction step.  Within every window of `window` consecutive
  * keys of a trace (1 <= window <= 4096) the keys are sorted by (evict_at, index).  Outputs, all int32
@@ -307,9 +307,10 @@ size_t kvs_host_arena_bytes(int batch, int total_tokens, int max_seqlen,
  * provides, >= kvs_host_arena_bytes(...), 256-byte aligned.  Returns the device status.
  * The work is pipelined over the Hkv KV-head groups, which are independent: while one group's
  * forward and backward run, the next group's inputs are uploaded and the previous group's results
- * downloaded, on two internal streams that (with their events) are created and destroyed inside
- * the call; no device memory is allocated.  The arena holds three groups at a time, so it is
- * smaller than the tensors when Hkv > 3.
+ * downloaded, on two internal streams that (with their events) are created on the first call on a
+ * device and reused by later calls until the process ends; no device memory is allocated.  Calls on
+ * the same device take turns.  The arena holds three groups at a time, so it is smaller than the
+ * tensors when Hkv > 3.
  */
 int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t* cu_seqlens_host,
                           const void* q_host, const void* k_host, const void* v_host,
@@ -321,7 +322,7 @@ int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t* cu_seqlen
                           void* arena, size_t arena_bytes, kvs_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
- * Rollout side (Sec. 1; Sec. 4 "Inference engine implementation"; App. A.3): the engine evicts KV
+ * Rollout side (Sec. 1; Sec. 4 "Inference engine implementation"; App. B.3): the engine evicts KV
  * entries directly in its paged cache and keeps decoding on the same stream.  Pages hold page_size
  * tokens (16 in one engine, with turns padded to page multiples; 1 in the other):
  *   k_cache, v_cache : bf16 [num_pages, page_size, Hkv, head_dim]

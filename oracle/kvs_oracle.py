@@ -25,13 +25,26 @@ What it states, and where that comes from:
 * Tile classes: the min/max rule per 128x128 tile and, independently, a brute
   force classification from the dense boolean mask.
 
+* Key slots: a trace's keys may be stored in any order if each slot carries the index and the
+  eviction step of the key it holds (``key_first``), e.g. sorted by eviction step for token-level
+  eviction (App. B.4), ``reorder_keys``; ``merge_partial`` is attention over a union of disjoint key sets.
+* ``dual_fwd``: student under the eviction mask + full-context teacher (self-distillation, App. D.3).
+* ``rope_rotate``: rotary embedding with positions that are never reset (Sec. 2).
+* ``dense_fwd_bwd_rounded`` / ``rounding_sigma``: the three bf16 roundings of the method (P, dS, the
+  stored O) switched on inside the fp64 definition, and their first-order propagation to a standard
+  deviation per output element: what the stated tolerances have to absorb.
+
 Everything is fp64 on inputs that were already rounded to bf16 by the caller.
-Pins (tests/test_oracle_pins.py, tests/test_mask_families.py): two-route agreement, no-eviction == plain
-causal attention (torch's CPU scaled_dot_product_attention in fp64), softmax
-rows summing to one, central finite differences for dQ/dK/dV, zero-query
-closed forms (exp(LSE) = live-key count, values printed in tests/golden),
-evict-after-one-step closed form, exact integer pair and tile counts.
-No function here is "parity unpinned".
+Pins (tests/test_oracle_pins.py, test_mask_families.py, test_oracle_rounding.py, test_key_slots.py,
+test_dual_forward.py, test_rope_and_packed.py): two-route agreement, no-eviction == plain causal
+attention (torch's CPU scaled_dot_product_attention in fp64), softmax rows summing to one, central
+finite differences for dQ/dK/dV (also through the rotation), zero-query closed forms (exp(LSE) =
+live-key count, values printed in tests/golden), evict-after-one-step closed form, exact integer pair and
+tile counts; key slots: invariance under key permutation, brute-force loops, rule vs brute-force
+classes; merge: student part + evicted part == full causal attention; rotation: plane rotation by hand,
+norm preservation, dependence on position differences only, inverse == transpose; rounding: roundings
+off == the dense definition bit for bit, the rounding helper against torch's bf16 conversion, the
+predicted deviation against the emulated error.  No function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -393,7 +406,7 @@ def evict_at_from_events(cu_seqlens, events):
 
 
 # --------------------------------------------------------------------------
-# paged KV cache with physical eviction (the engine's bookkeeping, Sec. 4 / App. A.3)
+# paged KV cache with physical eviction (the engine's bookkeeping, Sec. 4 / App. B.3)
 # --------------------------------------------------------------------------
 class PagedCacheModel:
     """Plain-Python model of the block tables and the free stack: pages of `page_size`
@@ -603,7 +616,7 @@ def reorder_keys(evict_at, window):
     (evict_at, index).  Returns perm (perm[s] = index of the key stored in slot s).  The slots then carry
     key_first = perm and key_evict = evict_at[perm]; the attention result is unchanged (sums over keys do
     not depend on their order), but the slots of a 128-slot block now leave the cache at about the same
-    time, which is what lets a tile be classified FULL or EMPTY (App. A.4 discusses token-level eviction)."""
+    time, which is what lets a tile be classified FULL or EMPTY (App. B.4 discusses token-level eviction)."""
     ev = np.asarray(evict_at, dtype=np.int64)
     T = ev.shape[0]
     perm = np.zeros(T, dtype=np.int64)

@@ -2,6 +2,7 @@
 #include <cudaTypedefs.h>
 
 #include "kvs_common.cuh"
+#include <mutex>
 #include <vector>
 
 namespace kvs {
@@ -131,6 +132,13 @@ extern "C" int kvs_selftest_bounded_wait(int32_t* status_word, int expected_arri
 // packed and unpacked by strided 2-D copies; the kernels run on a chunk as on any (Hq = G, Hkv = 1) problem.
 namespace {
 constexpr int HOST_SLOTS = 3;
+constexpr int kMaxHostDevices = 64;
+struct HostPipe {
+    cudaStream_t in = nullptr, outs = nullptr;
+    std::vector<cudaEvent_t> ev;
+};
+std::mutex g_host_mu[kMaxHostDevices];
+HostPipe g_host_pipe[kMaxHostDevices];
 // A slot's workspace status is reset by the next chunk that uses the slot; the first failure is kept here.
 __global__ void fold_status_kernel(const int32_t* ws_words, int32_t* sticky) {
     if (ws_words[1] != KVS_OK && *sticky == KVS_OK) *sticky = ws_words[1];
@@ -204,22 +212,20 @@ extern "C" int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t
     const int G = Hq / Hkv;
     const int NC = Hkv;                                    // chunks
     const size_t gsz = grad_dtype == KVS_GRAD_FP32 ? 4 : 2;
-    // Two copy streams and four events per chunk, all created and destroyed inside this call.
-    struct Res {
-        cudaStream_t in = nullptr, outs = nullptr;
-        std::vector<cudaEvent_t> ev;
-        ~Res() {
-            for (cudaEvent_t e : ev)
-                if (e) cudaEventDestroy(e);
-            if (in) cudaStreamDestroy(in);
-            if (outs) cudaStreamDestroy(outs);
-        }
-    } R;
-    if (cudaStreamCreateWithFlags(&R.in, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
-    if (cudaStreamCreateWithFlags(&R.outs, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
-    R.ev.assign((size_t)NC * 5 + 1, nullptr);
-    for (cudaEvent_t& e : R.ev)
+    // Two copy streams and five events per chunk.  They belong to the device, not to the call: created the first time
+    // the entry point runs on a device, reused by every later call (a trainer calls this once per layer and step) and
+    // kept until the process ends.  Calls on one device take turns (each ends with a synchronisation anyway).
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxHostDevices) return KVS_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_host_mu[dev]);
+    HostPipe& R = g_host_pipe[dev];
+    if (!R.in && cudaStreamCreateWithFlags(&R.in, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
+    if (!R.outs && cudaStreamCreateWithFlags(&R.outs, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
+    while (R.ev.size() < (size_t)NC * 5 + 1) {
+        cudaEvent_t e = nullptr;
         if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return KVS_ERR_CUDA;
+        R.ev.push_back(e);
+    }
     auto ev_qkv = [&](int c) { return R.ev[(size_t)c * 5 + 0]; };    // q, k, v of chunk c are on the device
     auto ev_dout = [&](int c) { return R.ev[(size_t)c * 5 + 1]; };   // dout of chunk c is on the device
     auto ev_fwd = [&](int c) { return R.ev[(size_t)c * 5 + 2]; };    // forward of chunk c done

@@ -2,7 +2,7 @@
 //
 // The inference engine of the method evicts KV entries directly in its paged cache (Sec. 1, Sec. 4
 // "Inference engine implementation": 16-token blocks in one engine, with completions padded to
-// block multiples (App. A.3); block size 1 in the other) and keeps decoding on the same stream.
+// block multiples (App. B.3); block size 1 in the other) and keeps decoding on the same stream.
 // Here: a block table per sequence lists the pages of its LIVE cache in order; eviction removes
 // whole pages from the table (the rows themselves never move) and returns them to a free list;
 // appending a token takes a page from the free list when the last page is full; decode attention

@@ -5,7 +5,7 @@ step ``evict_at`` that a compacting rollout would leave behind (Sec. 2,
 "KV-streams" paragraph: the trainer sees one continuous trace plus the spans
 the inference engine deleted) for the retention strategies of Sec. 3
 (Summary, Sliding Window / keep-last-k-turns) and for a token-level stress
-pattern (App. A.4 discusses token-level eviction), and it draws Gaussian
+pattern (App. B.4 discusses token-level eviction), and it draws Gaussian
 Q/K/V/dO.  None of the attention arithmetic lives here, so both the CPU
 oracle and the CUDA path may be fed from it.
 
@@ -146,7 +146,7 @@ def _turn_bounds(T: int, prompt: int, turn_lens):
 def markovian_thinker_events(T: int, prompt: int, turn_lens, budget: int):
     """Markovian Thinker (Sec. 3: o = B/2, s = 0): whenever the live context (prompt excluded)
     reaches ``budget`` tokens at the end of a turn, the oldest live turns are deleted until at
-    most half the budget remains.  Whole turns only (App. A.4).  Returns the event list."""
+    most half the budget remains.  Whole turns only (App. B.4).  Returns the event list."""
     starts, ends = _turn_bounds(T, prompt, turn_lens)
     live = []                       # indices of live turns, oldest first
     events = []

@@ -180,3 +180,57 @@ def test_full_size(name, kw):
     assert np.abs(n_gpu / live - 1.0).max() < 2e-4
     del out0, lse0
     torch.cuda.empty_cache()
+
+
+def test_full_size_token_level_with_reordered_keys():
+    # config 4 in the launch configuration bench.py times for its "keys re-ordered" line: window 4096, bf16 gradients.
+    # Checked against the oracle on sampled rows and on the metadata of every tile, and against the plain-order run of the
+    # same inputs (which test_full_size[cfg4] checks against the oracle) on every element.
+    w = W.make_workload(4, seed=0)
+    G = w.Hq // w.Hkv
+    rng = np.random.default_rng(12)
+    q, k, v, do = W.make_tensors(w, seed=0, device=DEV)
+    ev_d = torch.from_numpy(w.evict_at).to(DEV)
+    cu_d = torch.from_numpy(w.cu_seqlens).to(DEV)
+    Tt = w.total_tokens
+    perm, kf, ke = B.kvs_reorder_keys(ev_d, cu_d, w.max_seqlen, 4096)
+    ref_perm = O.reorder_keys(w.trace(0), 4096)
+    assert np.array_equal(perm.cpu().numpy(), ref_perm)
+    kp, vp = B.kvs_permute_rows(k, perm), B.kvs_permute_rows(v, perm)
+    meta = B.kvs_mask_meta_keys(kf, ke, cu_d, w.max_seqlen)
+    cls, kmin, kmax = B.kvs_mask_meta_export(meta, w.cu_seqlens, Tt, w.max_seqlen)
+    ref_cls = O.tile_classes_rule(w.evict_at[ref_perm], key_first=ref_perm)
+    assert np.array_equal(cls, ref_cls.ravel())
+    assert (ref_cls != O.EMPTY).sum() * 1.6 < 524800                      # 1.67x fewer tiles than the causal triangle
+    out, lse = B.kvs_attn_fwd(q, kp, vp, meta, w.batch, w.max_seqlen, w.softmax_scale)
+    ws = torch.empty(B.kvs_attn_bwd_workspace_bytes(Tt, w.Hq, w.Hkv, w.d, B.GRAD_BF16), dtype=torch.uint8, device=DEV)
+    dq, dkp, dvp = B.kvs_attn_bwd(do, q, kp, vp, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale, B.GRAD_BF16, workspace=ws)
+    assert B.kvs_device_status(meta) == B.KVS_OK and B.kvs_device_status(ws) == B.KVS_OK
+    dk, dv = B.kvs_permute_rows(dkp, perm, inverse=True), B.kvs_permute_rows(dvp, perm, inverse=True)
+    # sampled rows against the oracle
+    g_sel = int(rng.integers(0, w.Hkv))
+    ev = w.trace(0)
+    kb, vb = _np64(k[:, g_sel]), _np64(v[:, g_sel])
+    rows = _sample_rows(ev, rng, 40)
+    got_o, ref_o, got_l, ref_l, got_dq, ref_dq = [], [], [], [], [], []
+    for i in rows:
+        h = g_sel * G + int(rng.integers(0, G))
+        o, l, dqi, *_ = O.row_fwd_bwd(_np64(q[i, h]), kb, vb, _np64(do[i, h]), ev, i, w.scale)
+        ref_o.append(o); ref_l.append(l); ref_dq.append(dqi)
+        got_o.append(_np64(out[i, h])); got_l.append(float(lse[h, i])); got_dq.append(_np64(dq[i, h]))
+    _cmp("reordered out rows", np.stack(got_o), np.stack(ref_o))
+    _cmp("reordered lse rows", np.array(got_l), np.array(ref_l))
+    ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(np.stack(ref_dq)), 1e-30))) - 7)
+    assert (np.abs(np.stack(got_dq) - np.stack(ref_dq)) <= np.maximum(MAX_ABS, ulp)).all()
+    # every element against the plain key order
+    del kp, vp, dkp, dvp
+    meta0 = B.kvs_mask_meta(ev_d, cu_d, w.max_seqlen)
+    out0, lse0 = B.kvs_attn_fwd(q, k, v, meta0, w.batch, w.max_seqlen, w.softmax_scale)
+    dq0, dk0, dv0 = B.kvs_attn_bwd(do, q, k, v, out0, lse0, meta0, w.batch, w.max_seqlen, w.softmax_scale, B.GRAD_BF16, workspace=ws)
+    # two bf16 results of the same quantity, each within its own rounding of it
+    for name, a, b in (("out", out, out0), ("dq", dq, dq0), ("dk", dk, dk0), ("dv", dv, dv0)):
+        d = (a.float() - b.float()).abs()
+        tol = torch.clamp(2.0 ** (torch.floor(torch.log2(b.float().abs().clamp_min(1e-30))) - 6), min=MAX_ABS)
+        assert bool((d <= tol).all()), (name, float(d.max()))
+        assert float((a.float() - b.float()).norm() / b.float().norm()) <= REL_L2, name
+    assert float((lse - lse0).abs().max()) <= 1e-3

@@ -303,7 +303,9 @@ def run_per_config(torch, B, W, dev, peaks, gpu_index):
     """The other configurations on the same clock as the headline: 1 warm-up + 3 timed steps each."""
     res = {}
     for key, cfg, variant, reorder in (("0", 0, "", 0), ("1", 1, "", 0), ("3", 3, "", 0), ("4", 4, "", 0),
-                                       ("4_keys_reordered", 4, "", 4096), ("4_control", 4, "control", 0)):
+                                       ("4_keys_reordered", 4, "", 4096), ("4_control", 4, "control", 0),
+                                       ("4b", 4, "b", 0), ("4b_keys_reordered", 4, "b", 4096),
+                                       ("5", 5, "", 0), ("6", 6, "", 0), ("7", 7, "", 0)):
         w = W.make_workload(cfg, seed=0, variant=variant)
         sampler = ClockSampler(gpu_index)
         r = time_train_steps(torch, B, W, w, 0, dev, steps=3, warmup=1, grad=B.GRAD_BF16, sampler=sampler, reorder=reorder)

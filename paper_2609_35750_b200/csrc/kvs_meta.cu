@@ -100,6 +100,7 @@ __global__ void meta_minmax_kernel(const int32_t* __restrict__ evict_at, const i
         if (last > nb - 1) last = nb - 1;
         long long first = fmn / TILE;
         if (first > nb) first = nb;
+        if (first < 0) first = 0;                  // a negative key_first is reported below; never an index
         if (!key_first && !complement && last < n) last = n;
         col_first[warp] = (int32_t)first;
         col_last[warp] = (mx <= 0) ? -1 : (int32_t)last;

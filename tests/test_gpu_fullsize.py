@@ -234,3 +234,47 @@ def test_full_size_token_level_with_reordered_keys():
         assert bool((d <= tol).all()), (name, float(d.max()))
         assert float((a.float() - b.float()).norm() / b.float().norm()) <= REL_L2, name
     assert float((lse - lse0).abs().max()) <= 1e-3
+
+
+def test_full_size_student_and_teacher_forward():
+    # kvs_attn_fwd_dual on config 2 at full size (the call bench.py --path dual times): sampled rows of both streams
+    # against the oracle, the student stream against the plain forward bit for bit
+    w = W.make_workload(2, seed=0)
+    G = w.Hq // w.Hkv
+    rng = np.random.default_rng(13)
+    q, k, v, _ = W.make_tensors(w, seed=0, device=DEV, with_dout=False)
+    ev_d = torch.from_numpy(w.evict_at).to(DEV)
+    cu_d = torch.from_numpy(w.cu_seqlens).to(DEV)
+    meta = B.kvs_mask_meta(ev_d, cu_d, w.max_seqlen)
+    meta_e = B.kvs_mask_meta_evicted(ev_d, cu_d, w.max_seqlen)
+    os_, ls_, ot_, lt_ = B.kvs_attn_fwd_dual(q, k, v, meta, meta_e, w.batch, w.max_seqlen, w.softmax_scale)
+    assert B.kvs_device_status(meta) == B.KVS_OK and B.kvs_device_status(meta_e) == B.KVS_OK
+    out, lse = B.kvs_attn_fwd(q, k, v, meta, w.batch, w.max_seqlen, w.softmax_scale)
+    assert torch.equal(out, os_) and torch.equal(lse, ls_)
+    for b in range(w.batch):
+        a, e = int(w.cu_seqlens[b]), int(w.cu_seqlens[b + 1])
+        evb = w.trace(b)
+        inf = np.full(e - a, O.INF, dtype=np.int64)
+        g_sel = int(rng.integers(0, w.Hkv))
+        kb, vb = _np64(k[a:e, g_sel]), _np64(v[a:e, g_sel])
+        rows = _sample_rows(evb, rng, 24)
+        got_s, ref_s, got_t, ref_t, gl, rl = [], [], [], [], [], []
+        for i in rows:
+            h = g_sel * G + int(rng.integers(0, G))
+            o_s, l_s, _, _ = O.row_fwd(_np64(q[a + i, h]), kb, vb, evb, i, w.scale)
+            o_t, l_t, _, _ = O.row_fwd(_np64(q[a + i, h]), kb, vb, inf, i, w.scale)
+            ref_s.append(o_s); ref_t.append(o_t); rl += [l_s, l_t]
+            got_s.append(_np64(os_[a + i, h])); got_t.append(_np64(ot_[a + i, h])); gl += [float(ls_[h, a + i]), float(lt_[h, a + i])]
+        _cmp(f"trace {b} student rows", np.stack(got_s), np.stack(ref_s))
+        # the teacher is merged from two bf16 partial results: up to half an ulp more than a once-rounded output
+        ref_t = np.stack(ref_t)
+        ulp_half = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(ref_t), 1e-30))) - 8)
+        assert (np.abs(np.stack(got_t) - ref_t) <= MAX_ABS + ulp_half).all()
+        assert np.linalg.norm(np.stack(got_t) - ref_t) / np.linalg.norm(ref_t) <= REL_L2
+        _cmp(f"trace {b} lse rows", np.array(gl), np.array(rl))
+    # the teacher's normaliser counts every causal key: with q = 0, exp(lse_teacher) = i + 1
+    z = torch.zeros_like(q)
+    _, _, _, lt0 = B.kvs_attn_fwd_dual(z, k, v, meta, meta_e, w.batch, w.max_seqlen, w.softmax_scale)
+    n_gpu = torch.exp(lt0[0].double()).cpu().numpy()
+    want = np.concatenate([np.arange(1, int(w.cu_seqlens[b + 1] - w.cu_seqlens[b]) + 1) for b in range(w.batch)])
+    assert np.abs(n_gpu / want - 1.0).max() < 2e-4

@@ -65,3 +65,35 @@ def test_random_shapes_match_the_oracle(seed):
             nref = np.linalg.norm(ref)
             if nref > 1e-3:
                 assert np.linalg.norm(g - ref) / nref <= 5e-3, (name, what)
+
+
+def test_many_short_traces():
+    # a packed batch of 300 traces of 1..200 tokens: many block -> trace lookups, class matrices of one or two tiles,
+    # offsets that are rarely multiples of anything
+    from paper_2609_35750_b200 import binding as B
+    rng = np.random.default_rng(21)
+    lens = rng.integers(1, 201, size=300)
+    evs = []
+    for T in lens:
+        ev = np.full(T, int(W.INF), dtype=np.int64)
+        sel = rng.random(T) < 0.5
+        ev[sel] = (np.arange(T) + rng.integers(1, 60, size=T))[sel]
+        evs.append(ev.astype(np.int32))
+    cu = np.zeros(len(lens) + 1, dtype=np.int32)
+    cu[1:] = np.cumsum(lens)
+    w = W.Workload("many", cu, np.concatenate(evs), 4, 2, 64)
+    q, k, v, do = W.make_tensors(w, 21)
+    qd, kd, vd, dod = (t.cuda() for t in (q, k, v, do))
+    meta = B.kvs_mask_meta(torch.from_numpy(w.evict_at).cuda(), torch.from_numpy(w.cu_seqlens).cuda(), w.max_seqlen)
+    out, lse = B.kvs_attn_fwd(qd, kd, vd, meta, w.batch, w.max_seqlen, w.softmax_scale)
+    dq, dk, dv = B.kvs_attn_bwd(dod, qd, kd, vd, out, lse, meta, w.batch, w.max_seqlen, w.softmax_scale, B.GRAD_FP32)
+    assert B.kvs_device_status(meta) == B.KVS_OK
+    cls, kmin, kmax = B.kvs_mask_meta_export(meta, w.cu_seqlens, w.total_tokens, w.max_seqlen)
+    assert np.array_equal(cls, np.concatenate([O.tile_classes_rule(w.trace(b)).ravel() for b in range(w.batch)]))
+    f = lambda t: t.float().cpu().numpy().astype(np.float64)
+    ro, rl = O.varlen_fwd(f(q), f(k), f(v), w.evict_at, w.cu_seqlens, w.scale)
+    rdq, rdk, rdv = O.varlen_bwd(f(q), f(k), f(v), f(do), w.evict_at, w.cu_seqlens, w.scale)
+    for name, got, ref in (("out", out, ro), ("lse", lse, rl), ("dq", dq, rdq), ("dk", dk, rdk), ("dv", dv, rdv)):
+        g = f(got)
+        assert np.isfinite(g).all() and np.abs(g - ref).max() <= 2e-2, (name, float(np.abs(g - ref).max()))
+        assert np.linalg.norm(g - ref) / np.linalg.norm(ref) <= 5e-3, name

@@ -499,6 +499,7 @@ def main():
     ap.add_argument("--path", type=str, default="train", choices=["train", "meta", "decode", "dual"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e", action="store_true", help="measure the host-buffer entry point also when the case was reduced by a flag")
     ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--shrink", type=int, default=1, help="divide every length of the configuration (small cases for profilers)")
@@ -573,7 +574,7 @@ def main():
 
     # ---- end to end through the C ABI with host buffers ------------------------------------------
     e2e = None
-    if not args.no_e2e and not small:
+    if not args.no_e2e and (not small or args.e2e):
         pin = lambda t: t.cpu().contiguous().pin_memory()
         hq, hk, hv, hdo = pin(q), pin(k), pin(v), pin(do)
         hev, hcu = pin(torch.from_numpy(w.evict_at)), pin(torch.from_numpy(w.cu_seqlens))

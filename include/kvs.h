@@ -305,12 +305,15 @@ size_t kvs_host_arena_bytes(int batch, int total_tokens, int max_seqlen,
  * backward, copies out, lse, dq, dk, dv back, and SYNCHRONISES the stream.  Host buffers
  * should be page-locked for the copies to be asynchronous.  arena: device memory the caller
  * provides, >= kvs_host_arena_bytes(...), 256-byte aligned.  Returns the device status.
- * The work is pipelined over the Hkv KV-head groups, which are independent: while one group's
- * forward and backward run, the next group's inputs are uploaded and the previous group's results
- * downloaded, on two internal streams that (with their events) are created on the first call on a
- * device and reused by later calls until the process ends; no device memory is allocated.  Calls on
- * the same device take turns.  The arena holds three groups at a time, so it is smaller than the
- * tensors when Hkv > 3.
+ * The work is pipelined over chunks of (a contiguous range of traces, one KV-head group), which are
+ * independent: while one chunk's forward and backward run, the next chunk's inputs are uploaded and
+ * the previous chunk's results downloaded, on two internal streams that (with their events) are
+ * created on the first call on a device and reused by later calls until the process ends; no device
+ * memory is allocated.  With Hkv >= 8 a chunk is one KV-head group over all tokens; with fewer KV
+ * heads the batch is cut into ceil(8 / Hkv) trace ranges of about equal token counts (at most one per
+ * trace), each with mask metadata of its own.  Calls on the same device take turns.  The arena holds
+ * three chunks at a time, so it is smaller than the tensors when there are more than three.
+ * cu_seqlens_host is checked on the host before anything is queued (KVS_ERR_INVALID_ARG).
  */
 int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t* cu_seqlens_host,
                           const void* q_host, const void* k_host, const void* v_host,

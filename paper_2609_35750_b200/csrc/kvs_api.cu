@@ -125,58 +125,81 @@ extern "C" int kvs_selftest_bounded_wait(int32_t* status_word, int expected_arri
 }
 
 // ---- whole path from host buffers ------------------------------------------------------------
-// The work is cut into one chunk per KV head (its G query heads, all tokens): chunks are independent
-// in the forward and the backward, so while chunk c computes, the inputs of chunk c+1 arrive and
-// the results of chunk c-1 leave (PCIe is full duplex; two copy streams besides the caller's).
-// Each chunk lives in one of HOST_SLOTS sets of contiguous [tokens, G, d] / [tokens, 1, d] buffers,
-// packed and unpacked by strided 2-D copies; the kernels run on a chunk as on any (Hq = G, Hkv = 1) problem.
+// The work is cut into chunks of (a contiguous range of traces, one KV head with its G query heads): chunks are
+// independent in the forward and the backward, so while chunk c computes, the inputs of chunk c+1 arrive and
+// the results of chunk c-1 leave (PCIe is full duplex; two copy streams besides the caller's).  What cannot
+// overlap is the first chunk's upload and the last chunk's download, so the batch is cut into as many trace
+// ranges as it takes to have about HOST_TARGET_CHUNKS chunks.  Every range gets mask metadata of its own
+// (its traces re-based to token 0).  Each chunk lives in one of HOST_SLOTS sets of contiguous
+// [tokens, G, d] / [tokens, 1, d] buffers, packed and unpacked by strided 2-D copies; the kernels run on a
+// chunk as on any (Hq = G, Hkv = 1) problem.
 namespace {
-constexpr int HOST_SLOTS = 3;
+#ifndef KVS_HOST_SLOTS
+#define KVS_HOST_SLOTS 3
+#endif
+#ifndef KVS_HOST_CHUNKS
+#define KVS_HOST_CHUNKS 8
+#endif
+constexpr int HOST_SLOTS = KVS_HOST_SLOTS;
+constexpr int HOST_TARGET_CHUNKS = KVS_HOST_CHUNKS;
 constexpr int kMaxHostDevices = 64;
 struct HostPipe {
     cudaStream_t in = nullptr, outs = nullptr;
     std::vector<cudaEvent_t> ev;
+    std::vector<int32_t> cu_ranges;          // re-based cu_seqlens of the trace ranges (staging for one upload)
 };
 std::mutex g_host_mu[kMaxHostDevices];
 HostPipe g_host_pipe[kMaxHostDevices];
-// A slot's workspace status is reset by the next chunk that uses the slot; the first failure is kept here.
-__global__ void fold_status_kernel(const int32_t* ws_words, int32_t* sticky) {
-    if (ws_words[1] != KVS_OK && *sticky == KVS_OK) *sticky = ws_words[1];
+
+// A slot's workspace status and a range's metadata status are folded into one sticky word: one failure is kept.
+__global__ void fold_status_kernel(const int32_t* words, int32_t* sticky) {
+    if (words[1] != KVS_OK) atomicCAS(sticky, KVS_OK, words[1]);
 }
+
+inline int host_ranges(int batch, int Hkv) {
+    int r = (HOST_TARGET_CHUNKS + Hkv - 1) / Hkv;
+    if (r > batch) r = batch;
+    return r < 1 ? 1 : r;
+}
+
 struct ArenaLayout {
     size_t evict, cu, sticky, meta, slot0, slot_stride, total;      // global part, then HOST_SLOTS equal slots
-    size_t q, k, v, dout, out, lse, dq, dk, dv, ws;          // offsets inside a slot
-    size_t meta_bytes, ws_bytes, nq_bytes, nkv_bytes, gq_bytes, gkv_bytes, lse_bytes;   // per chunk
-    int slots;
+    size_t q, k, v, dout, out, lse, dq, dk, dv, ws;                  // offsets inside a slot
+    size_t meta_stride, ws_bytes;
+    int slots, ranges, slot_tokens;
 };
 ArenaLayout arena_layout(int batch, int total_tokens, int max_seqlen, int Hq, int Hkv, int head_dim, int grad_dtype) {
     ArenaLayout A;
     const int G = Hq / Hkv;
     const size_t gsz = grad_dtype == KVS_GRAD_FP32 ? 4 : 2;
-    A.slots = Hkv < HOST_SLOTS ? Hkv : HOST_SLOTS;
-    A.nq_bytes = (size_t)total_tokens * G * head_dim * 2;
-    A.nkv_bytes = (size_t)total_tokens * head_dim * 2;
-    A.gq_bytes = (size_t)total_tokens * G * head_dim * gsz;
-    A.gkv_bytes = (size_t)total_tokens * head_dim * gsz;
-    A.lse_bytes = (size_t)total_tokens * G * 4;
-    A.meta_bytes = kvs_mask_meta_bytes(batch, total_tokens, max_seqlen);
-    A.ws_bytes = kvs_attn_bwd_workspace_bytes(total_tokens, G, 1, head_dim, grad_dtype);
+    if (max_seqlen > total_tokens) max_seqlen = total_tokens;
+    A.ranges = host_ranges(batch, Hkv);
+    const long long nchunks = (long long)A.ranges * Hkv;
+    A.slots = nchunks < HOST_SLOTS ? (int)nchunks : HOST_SLOTS;
+    // a range is closed as soon as it holds its share of the tokens, so it exceeds the share by less than one trace
+    long long st = (long long)total_tokens / A.ranges + max_seqlen;
+    if (st > total_tokens) st = total_tokens;
+    A.slot_tokens = (int)st;
+    const size_t nq = (size_t)st * G * head_dim * 2, nkv = (size_t)st * head_dim * 2;
+    const size_t gq = (size_t)st * G * head_dim * gsz, gkv = (size_t)st * head_dim * gsz;
+    A.meta_stride = align_up(kvs_mask_meta_bytes(batch, A.slot_tokens, max_seqlen), 256);
+    A.ws_bytes = kvs_attn_bwd_workspace_bytes(A.slot_tokens, G, 1, head_dim, grad_dtype);
     size_t o = 0;
     A.evict = o; o = align_up(o + (size_t)total_tokens * 4, 256);
-    A.cu = o;    o = align_up(o + (size_t)(batch + 1) * 4, 256);
+    A.cu = o;    o = align_up(o + (size_t)(batch + A.ranges) * 4, 256);
     A.sticky = o; o += 256;
-    A.meta = o;  o = align_up(o + A.meta_bytes, 256);
+    A.meta = o;  o += (size_t)A.ranges * A.meta_stride;
     A.slot0 = o;
     size_t t = 0;
-    A.q = t;     t = align_up(t + A.nq_bytes, 256);
-    A.k = t;     t = align_up(t + A.nkv_bytes, 256);
-    A.v = t;     t = align_up(t + A.nkv_bytes, 256);
-    A.dout = t;  t = align_up(t + A.nq_bytes, 256);
-    A.out = t;   t = align_up(t + A.nq_bytes, 256);
-    A.lse = t;   t = align_up(t + A.lse_bytes, 256);
-    A.dq = t;    t = align_up(t + A.gq_bytes, 256);
-    A.dk = t;    t = align_up(t + A.gkv_bytes, 256);
-    A.dv = t;    t = align_up(t + A.gkv_bytes, 256);
+    A.q = t;     t = align_up(t + nq, 256);
+    A.k = t;     t = align_up(t + nkv, 256);
+    A.v = t;     t = align_up(t + nkv, 256);
+    A.dout = t;  t = align_up(t + nq, 256);
+    A.out = t;   t = align_up(t + nq, 256);
+    A.lse = t;   t = align_up(t + (size_t)st * G * 4, 256);
+    A.dq = t;    t = align_up(t + gq, 256);
+    A.dk = t;    t = align_up(t + gkv, 256);
+    A.dv = t;    t = align_up(t + gkv, 256);
     A.ws = t;    t = align_up(t + A.ws_bytes, 256);
     A.slot_stride = t;
     A.total = A.slot0 + (size_t)A.slots * A.slot_stride;
@@ -188,6 +211,7 @@ extern "C" size_t kvs_host_arena_bytes(int batch, int total_tokens, int max_seql
     if (batch < 0 || total_tokens < 0 || max_seqlen < 0 || Hq <= 0 || Hkv <= 0 || head_dim <= 0) return 0;
     if (Hq % Hkv != 0) return 0;
     if (grad_dtype != KVS_GRAD_BF16 && grad_dtype != KVS_GRAD_FP32) return 0;
+    if (batch == 0 || total_tokens == 0) return 256;
     return arena_layout(batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, grad_dtype).total;
 }
 
@@ -205,12 +229,18 @@ extern "C" int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t
         !dk_host || !dv_host || !arena)
         return KVS_ERR_INVALID_ARG;
     if (((uintptr_t)arena & 255) != 0) return KVS_ERR_ALIGNMENT;
+    if (max_seqlen > total_tokens) max_seqlen = total_tokens;
+    // cu_seqlens is a host array here, so it can be checked before anything is queued
+    if (cu_seqlens_host[0] != 0 || cu_seqlens_host[batch] != total_tokens) return KVS_ERR_INVALID_ARG;
+    for (int b = 0; b < batch; ++b) {
+        const long long T = (long long)cu_seqlens_host[b + 1] - cu_seqlens_host[b];
+        if (T < 0 || T > max_seqlen) return KVS_ERR_INVALID_ARG;
+    }
     const ArenaLayout A = arena_layout(batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, grad_dtype);
     if (arena_bytes < A.total) return KVS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     char* a = (char*)arena;
     const int G = Hq / Hkv;
-    const int NC = Hkv;                                    // chunks
     const size_t gsz = grad_dtype == KVS_GRAD_FP32 ? 4 : 2;
     // Two copy streams and five events per chunk.  They belong to the device, not to the call: created the first time
     // the entry point runs on a device, reused by every later call (a trainer calls this once per layer and step) and
@@ -221,6 +251,40 @@ extern "C" int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t
     HostPipe& R = g_host_pipe[dev];
     if (!R.in && cudaStreamCreateWithFlags(&R.in, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
     if (!R.outs && cudaStreamCreateWithFlags(&R.outs, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
+
+    // trace ranges: contiguous, each closed once it holds its share of the tokens
+    struct Range { int b0, b1, tok0, tokens, maxlen, cu_off; };
+    std::vector<Range> ranges;
+    R.cu_ranges.clear();
+    {
+        const long long share = ((long long)total_tokens + A.ranges - 1) / A.ranges;
+        int b = 0;
+        while (b < batch) {
+            Range r;
+            r.b0 = b;
+            r.tok0 = cu_seqlens_host[b];
+            r.maxlen = 0;
+            r.cu_off = (int)R.cu_ranges.size();
+            R.cu_ranges.push_back(0);
+            const int left_ranges = A.ranges - (int)ranges.size();      // >= 1: the last one takes all that is left
+            while (b < batch) {
+                const int T = cu_seqlens_host[b + 1] - cu_seqlens_host[b];
+                R.cu_ranges.push_back(cu_seqlens_host[b + 1] - r.tok0);
+                if (T > r.maxlen) r.maxlen = T;
+                ++b;
+                const bool last_range = left_ranges <= 1;
+                if (!last_range && ((long long)cu_seqlens_host[b] - r.tok0 >= share || batch - b <= left_ranges - 1)) break;
+            }
+            r.b1 = b;
+            r.tokens = cu_seqlens_host[b] - r.tok0;
+            if (r.tokens > 0) ranges.push_back(r);          // a range of empty traces has no rows to compute or copy
+            else R.cu_ranges.resize(r.cu_off);
+        }
+    }
+    const int NR = (int)ranges.size();
+    for (const Range& r : ranges)
+        if (r.tokens > A.slot_tokens) return KVS_ERR_WORKSPACE;      // cannot happen: see arena_layout
+    const int NC = NR * Hkv;                                          // chunk c = (range c / Hkv, KV head c % Hkv)
     while (R.ev.size() < (size_t)NC * 5 + 1) {
         cudaEvent_t e = nullptr;
         if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return KVS_ERR_CUDA;
@@ -234,71 +298,82 @@ extern "C" int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t
     cudaEvent_t ev_start = R.ev[(size_t)NC * 5];
 #define KVS_CK(call) \
     if ((call) != cudaSuccess) return KVS_ERR_CUDA
-    // rows of `width` bytes, `tokens` of them: host row pitch hp, device row pitch = width
-    auto h2d = [&](cudaStream_t s_, void* dst, const void* src, size_t hoff, size_t hp, size_t width) {
-        return cudaMemcpy2DAsync(dst, width, (const char*)src + hoff, hp, width, (size_t)total_tokens, cudaMemcpyHostToDevice, s_);
-    };
-    auto d2h = [&](cudaStream_t s_, void* dst, size_t hoff, size_t hp, const void* src, size_t width) {
-        return cudaMemcpy2DAsync((char*)dst + hoff, hp, src, width, width, (size_t)total_tokens, cudaMemcpyDeviceToHost, s_);
-    };
     KVS_CK(cudaMemcpyAsync(a + A.evict, evict_at_host, (size_t)total_tokens * 4, cudaMemcpyHostToDevice, st));
-    KVS_CK(cudaMemcpyAsync(a + A.cu, cu_seqlens_host, (size_t)(batch + 1) * 4, cudaMemcpyHostToDevice, st));
+    KVS_CK(cudaMemcpyAsync(a + A.cu, R.cu_ranges.data(), R.cu_ranges.size() * 4, cudaMemcpyHostToDevice, st));
     KVS_CK(cudaMemsetAsync(a + A.sticky, 0, 4, st));
-    KVS_CK(cudaEventRecord(ev_start, st));                 // the copy streams start after what the caller queued before
+    int rc = KVS_OK;
+    for (int r = 0; r < NR; ++r) {
+        const Range& g = ranges[r];
+        char* meta = a + A.meta + (size_t)r * A.meta_stride;
+        rc = kvs_mask_meta((const int32_t*)(a + A.evict) + g.tok0, (const int32_t*)(a + A.cu) + g.cu_off, g.b1 - g.b0, g.tokens, g.maxlen,
+                           meta, A.meta_stride, stream);
+        if (rc != KVS_OK) return rc;
+    }
+    KVS_CK(cudaEventRecord(ev_start, st));                 // the internal streams start after what the caller queued before
     KVS_CK(cudaStreamWaitEvent(R.in, ev_start, 0));
     KVS_CK(cudaStreamWaitEvent(R.outs, ev_start, 0));
-    int rc = kvs_mask_meta((const int32_t*)(a + A.evict), (const int32_t*)(a + A.cu), batch, total_tokens, max_seqlen, a + A.meta,
-                           A.meta_bytes, stream);
-    if (rc != KVS_OK) return rc;
     const size_t hq_pitch = (size_t)Hq * head_dim * 2, hkv_pitch = (size_t)Hkv * head_dim * 2;
     const size_t wq = (size_t)G * head_dim * 2, wkv = (size_t)head_dim * 2;
     const size_t gq_pitch = (size_t)Hq * head_dim * gsz, gkv_pitch = (size_t)Hkv * head_dim * gsz;
     const size_t wgq = (size_t)G * head_dim * gsz, wgkv = (size_t)head_dim * gsz;
+    // rows of `width` bytes, one per token of the chunk's range: host row pitch hp, device row pitch = width
+    auto h2d = [&](cudaStream_t s_, void* dst, const void* src, size_t hoff, size_t hp, size_t width, const Range& g) {
+        return cudaMemcpy2DAsync(dst, width, (const char*)src + (size_t)g.tok0 * hp + hoff, hp, width, (size_t)g.tokens,
+                                 cudaMemcpyHostToDevice, s_);
+    };
+    auto d2h = [&](cudaStream_t s_, void* dst, size_t hoff, size_t hp, const void* src, size_t width, const Range& g) {
+        return cudaMemcpy2DAsync((char*)dst + (size_t)g.tok0 * hp + hoff, hp, src, width, width, (size_t)g.tokens,
+                                 cudaMemcpyDeviceToHost, s_);
+    };
     auto upload = [&](int c) -> int {
+        const Range& g = ranges[c / Hkv];
+        const int kh = c % Hkv;
         char* sl = a + A.slot0 + (size_t)(c % A.slots) * A.slot_stride;
         if (c >= A.slots) KVS_CK(cudaStreamWaitEvent(R.in, ev_down(c - A.slots), 0));     // the slot's previous chunk is finished
-        KVS_CK(h2d(R.in, sl + A.q, q_host, (size_t)c * wq, hq_pitch, wq));
-        KVS_CK(h2d(R.in, sl + A.k, k_host, (size_t)c * wkv, hkv_pitch, wkv));
-        KVS_CK(h2d(R.in, sl + A.v, v_host, (size_t)c * wkv, hkv_pitch, wkv));
+        KVS_CK(h2d(R.in, sl + A.q, q_host, (size_t)kh * wq, hq_pitch, wq, g));
+        KVS_CK(h2d(R.in, sl + A.k, k_host, (size_t)kh * wkv, hkv_pitch, wkv, g));
+        KVS_CK(h2d(R.in, sl + A.v, v_host, (size_t)kh * wkv, hkv_pitch, wkv, g));
         KVS_CK(cudaEventRecord(ev_qkv(c), R.in));
-        KVS_CK(h2d(R.in, sl + A.dout, dout_host, (size_t)c * wq, hq_pitch, wq));
+        KVS_CK(h2d(R.in, sl + A.dout, dout_host, (size_t)kh * wq, hq_pitch, wq, g));
         KVS_CK(cudaEventRecord(ev_dout(c), R.in));
         return KVS_OK;
     };
     for (int c = 0; c < A.slots && c < NC; ++c)
         if ((rc = upload(c)) != KVS_OK) return rc;
     for (int c = 0; c < NC; ++c) {
+        const Range& g = ranges[c / Hkv];
+        const int kh = c % Hkv, nb = g.b1 - g.b0;
         char* sl = a + A.slot0 + (size_t)(c % A.slots) * A.slot_stride;
+        char* meta = a + A.meta + (size_t)(c / Hkv) * A.meta_stride;
         KVS_CK(cudaStreamWaitEvent(st, ev_qkv(c), 0));
-        rc = kvs_attn_fwd(sl + A.q, sl + A.k, sl + A.v, a + A.meta, batch, total_tokens, max_seqlen, G, 1, head_dim, softmax_scale,
-                          sl + A.out, (float*)(sl + A.lse), stream);
+        rc = kvs_attn_fwd(sl + A.q, sl + A.k, sl + A.v, meta, nb, g.tokens, g.maxlen, G, 1, head_dim, softmax_scale, sl + A.out,
+                          (float*)(sl + A.lse), stream);
         if (rc != KVS_OK) return rc;
         KVS_CK(cudaEventRecord(ev_fwd(c), st));
         KVS_CK(cudaStreamWaitEvent(R.outs, ev_fwd(c), 0));
-        KVS_CK(d2h(R.outs, out_host, (size_t)c * wq, hq_pitch, sl + A.out, wq));
-        KVS_CK(cudaMemcpyAsync((char*)lse_host + (size_t)c * A.lse_bytes, sl + A.lse, A.lse_bytes, cudaMemcpyDeviceToHost, R.outs));
+        KVS_CK(d2h(R.outs, out_host, (size_t)kh * wq, hq_pitch, sl + A.out, wq, g));
+        // lse: G rows of the range's tokens, host rows total_tokens apart
+        KVS_CK(cudaMemcpy2DAsync((char*)lse_host + ((size_t)kh * G * total_tokens + g.tok0) * 4, (size_t)total_tokens * 4, sl + A.lse,
+                                 (size_t)g.tokens * 4, (size_t)g.tokens * 4, (size_t)G, cudaMemcpyDeviceToHost, R.outs));
         KVS_CK(cudaStreamWaitEvent(st, ev_dout(c), 0));
-        rc = kvs_attn_bwd(sl + A.dout, sl + A.q, sl + A.k, sl + A.v, sl + A.out, (const float*)(sl + A.lse), a + A.meta, batch,
-                          total_tokens, max_seqlen, G, 1, head_dim, softmax_scale, grad_dtype, sl + A.dq, sl + A.dk, sl + A.dv,
-                          sl + A.ws, A.ws_bytes, stream);
+        rc = kvs_attn_bwd(sl + A.dout, sl + A.q, sl + A.k, sl + A.v, sl + A.out, (const float*)(sl + A.lse), meta, nb, g.tokens, g.maxlen,
+                          G, 1, head_dim, softmax_scale, grad_dtype, sl + A.dq, sl + A.dk, sl + A.dv, sl + A.ws, A.ws_bytes, stream);
         if (rc != KVS_OK) return rc;
         fold_status_kernel<<<1, 1, 0, st>>>((const int32_t*)(sl + A.ws), (int32_t*)(a + A.sticky));
+        if (kh == Hkv - 1) fold_status_kernel<<<1, 1, 0, st>>>((const int32_t*)meta, (int32_t*)(a + A.sticky));
         KVS_CK(cudaEventRecord(ev_bwd(c), st));
         KVS_CK(cudaStreamWaitEvent(R.outs, ev_bwd(c), 0));
-        KVS_CK(d2h(R.outs, dq_host, (size_t)c * wgq, gq_pitch, sl + A.dq, wgq));
-        KVS_CK(d2h(R.outs, dk_host, (size_t)c * wgkv, gkv_pitch, sl + A.dk, wgkv));
-        KVS_CK(d2h(R.outs, dv_host, (size_t)c * wgkv, gkv_pitch, sl + A.dv, wgkv));
+        KVS_CK(d2h(R.outs, dq_host, (size_t)kh * wgq, gq_pitch, sl + A.dq, wgq, g));
+        KVS_CK(d2h(R.outs, dk_host, (size_t)kh * wgkv, gkv_pitch, sl + A.dk, wgkv, g));
+        KVS_CK(d2h(R.outs, dv_host, (size_t)kh * wgkv, gkv_pitch, sl + A.dv, wgkv, g));
         KVS_CK(cudaEventRecord(ev_down(c), R.outs));
         if (c + A.slots < NC && (rc = upload(c + A.slots)) != KVS_OK) return rc;
     }
     KVS_CK(cudaStreamWaitEvent(st, ev_down(NC - 1), 0));   // the caller's stream ends after every copy (the out stream is in order)
 #undef KVS_CK
-    // status words: the metadata buffer's (mask validation, forward) and the folded workspace status (backward)
-    int32_t hm[2] = {0, 0}, hs = 0;
-    if (cudaMemcpyAsync(hm, a + A.meta, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVS_ERR_CUDA;
+    // the sticky word holds the first failure of any range's metadata (mask validation, forward) or workspace (backward)
+    int32_t hs = 0;
     if (cudaMemcpyAsync(&hs, a + A.sticky, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVS_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return KVS_ERR_CUDA;
-    if (hm[1] != KVS_OK) return hm[1];
-    if (hs != KVS_OK) return hs;
-    return KVS_OK;
+    return hs;
 }

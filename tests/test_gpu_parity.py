@@ -310,18 +310,26 @@ def test_argument_errors():
     assert e.value.code == B.KVS_ERR_ALIGNMENT
 
 
-@pytest.mark.parametrize("Hq,Hkv,grad", [(4, 2, "bf16"), (10, 5, "bf16"), (3, 1, "fp32"), (8, 4, "fp32")])
-def test_host_buffer_entry_point_matches_device_path(Hq, Hkv, grad):
-    # the host path pipelines over KV-head groups (three in flight): more groups than slots, a single group,
-    # both gradient types; every group must come back exactly as the one-shot device path computes it
+@pytest.mark.parametrize("Hq,Hkv,grad,batch,empty", [(4, 2, "bf16", 3, ()), (10, 5, "bf16", 3, ()), (3, 1, "fp32", 3, ()), (8, 4, "fp32", 3, ()),
+                                                      (16, 8, "bf16", 11, ()), (2, 1, "bf16", 1, ()), (8, 8, "fp32", 9, (0, 4, 5, 8))])
+def test_host_buffer_entry_point_matches_device_path(Hq, Hkv, grad, batch, empty):
+    # the host path pipelines over chunks of (a range of traces, one KV-head group), three in flight, each range with mask
+    # metadata of its own: one trace per range, several ragged traces per range, a single trace, ranges that meet empty
+    # traces, both gradient types; every chunk must come back exactly as the one-shot device path computes it
     grad = B.GRAD_BF16 if grad == "bf16" else B.GRAD_FP32
-    w = W.make_workload(3, shrink=32, Hq=Hq, Hkv=Hkv, batch=3)
+    w = W.make_workload(3, shrink=32, Hq=Hq, Hkv=Hkv, batch=batch - len(empty))
+    if empty:                                            # splice zero-length traces into the packed batch
+        lens = np.diff(w.cu_seqlens).tolist()
+        for b in empty:
+            lens.insert(b, 0)
+        w.cu_seqlens = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        assert w.batch == batch
     q, k, v, do = W.make_tensors(w, 9)
     qd, kd, vd, dod = (t.to(DEV) for t in (q, k, v, do))
     _, out, lse, dq, dk, dv = _run_gpu(w, qd, kd, vd, dod, grad)
     pin = lambda t: t.contiguous().pin_memory()
     gdt = torch.bfloat16 if grad == B.GRAD_BF16 else torch.float32
-    ho, hl = pin(torch.empty_like(q)), pin(torch.empty((w.Hq, w.total_tokens), dtype=torch.float32))
+    ho, hl = pin(torch.full(q.shape, float("nan"), dtype=q.dtype)), pin(torch.full((w.Hq, w.total_tokens), float("nan")))
     hdq, hdk, hdv = (pin(torch.full(t.shape, float("nan"), dtype=gdt)) for t in (q, k, v))
     arena = torch.empty(B.kvs_host_arena_bytes(w.batch, w.total_tokens, w.max_seqlen, w.Hq, w.Hkv, w.d, grad),
                         dtype=torch.uint8, device=DEV)
@@ -330,6 +338,36 @@ def test_host_buffer_entry_point_matches_device_path(Hq, Hkv, grad):
     assert torch.equal(ho, out.cpu()) and torch.equal(hl, lse.cpu())
     assert torch.equal(hdk, dk.cpu()) and torch.equal(hdv, dv.cpu())
     assert torch.allclose(hdq.float(), dq.cpu().float(), atol=2e-2, rtol=2e-2)
+
+
+def test_host_buffer_entry_point_reports_bad_masks_and_bad_trace_tables():
+    # a malformed cu_seqlens is refused on the host; a key evicted before its own step in the LAST trace range is seen by
+    # that range's metadata pass on the device and comes back as the call's status; the arena is usable afterwards
+    w = W.make_workload(3, shrink=32, Hq=4, Hkv=2, batch=5)
+    q, k, v, do = W.make_tensors(w, 2)
+    pin = lambda t: t.contiguous().pin_memory()
+    hq, hk, hv, hdo = pin(q), pin(k), pin(v), pin(do)
+    outs = lambda: (pin(torch.empty_like(q)), pin(torch.empty((w.Hq, w.total_tokens))), pin(torch.empty_like(q)), pin(torch.empty_like(k)),
+                    pin(torch.empty_like(v)))
+    arena = torch.empty(B.kvs_host_arena_bytes(w.batch, w.total_tokens, w.max_seqlen, w.Hq, w.Hkv, w.d, B.GRAD_BF16),
+                        dtype=torch.uint8, device=DEV)
+    call = lambda ev, cu, o: B.kvs_attn_fwd_bwd_host(pin(torch.from_numpy(ev)), pin(torch.from_numpy(cu)), hq, hk, hv, hdo, w.max_seqlen,
+                                                     w.softmax_scale, B.GRAD_BF16, *o, arena)
+    for bad_cu in (np.concatenate([w.cu_seqlens[:-1], [w.total_tokens - 1]]),                       # does not end at total_tokens
+                   np.concatenate([w.cu_seqlens[:2], [w.cu_seqlens[1] - 1], w.cu_seqlens[3:]])):   # a negative length
+        with pytest.raises(B.KvsError) as e:
+            call(w.evict_at, bad_cu.astype(np.int32), outs())
+        assert e.value.code == B.KVS_ERR_INVALID_ARG
+    bad_ev = w.evict_at.copy()
+    j = int(w.cu_seqlens[-2]) + 77                       # key 77 of the last trace
+    bad_ev[j] = 77
+    with pytest.raises(B.KvsError) as e:
+        call(bad_ev, w.cu_seqlens, outs())
+    assert e.value.code == B.KVS_ERR_BAD_EVICT
+    good = outs()
+    call(w.evict_at, w.cu_seqlens, good)
+    _, out, lse, _, dk, _ = _run_gpu(w, *(t.to(DEV) for t in (q, k, v, do)), B.GRAD_BF16)
+    assert torch.equal(good[0], out.cpu()) and torch.equal(good[1], lse.cpu()) and torch.equal(good[3], dk.cpu())
 
 
 # ---- the error of the CUDA path is the method's own operand rounding -------------------------------

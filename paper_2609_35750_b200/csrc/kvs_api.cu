@@ -57,6 +57,19 @@ int make_tmap_f32_thd(CUtensorMap* map, const void* base, int total_tokens, int 
     return r == CUDA_SUCCESS ? KVS_OK : KVS_ERR_CUDA;
 }
 
+int make_tmap_rows(CUtensorMap* map, const void* base, int rows, int cols) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return KVS_ERR_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {64, 1};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? KVS_OK : KVS_ERR_CUDA;
+}
+
 int check_device_sm100() {
     int dev = 0, major = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return KVS_ERR_CUDA;

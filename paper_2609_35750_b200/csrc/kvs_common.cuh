@@ -133,6 +133,9 @@ struct WsHeader {
 int make_tmap_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows, long long token_stride = 0);
 int make_tmap_f32_thd(CUtensorMap* map, const void* base, int total_tokens, int heads, int head_dim, int box_rows,
                       long long token_stride = 0);
+// bf16 [rows, cols] as a 2-D tensor whose box is 64 columns of ONE row: the form TMA gather4 takes (four row
+// coordinates per instruction), 128-byte swizzle
+int make_tmap_rows(CUtensorMap* map, const void* base, int rows, int cols);
 int check_device_sm100();
 
 #ifdef __CUDACC__

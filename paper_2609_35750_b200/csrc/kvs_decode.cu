@@ -32,6 +32,7 @@ struct DecodeParams {
     const int32_t* block_table;      // [S, max_pages]
     const int32_t* n_tokens;         // [S]
     int S, Hq, Hkv, page_size, max_pages, num_pages, nsplit;
+    int page_shift;                  // log2(page_size) when it is a power of two, else -1
     int32_t* status;                 // workspace status word: a page id outside [0, num_pages) is recorded there
     float scale_log2;
     float* part_o;                   // [S, Hq, nsplit, D] unnormalised
@@ -40,6 +41,16 @@ struct DecodeParams {
 
 // A block-table entry is only followed if it names a page of the cache: anything else (a stale or
 // corrupt table) is recorded as KVS_ERR_INVALID_ARG and read as page 0, so no kernel reads outside the cache.
+// token index -> (entry of the block table, row inside the page) without a division for power-of-two pages
+__device__ __forceinline__ void split_token(const DecodeParams& p, int tok, int& entry, int& offset) {
+    if (p.page_shift >= 0) {
+        entry = tok >> p.page_shift;
+        offset = tok & (p.page_size - 1);
+    } else {
+        entry = tok / p.page_size;
+        offset = tok - entry * p.page_size;
+    }
+}
 __device__ __forceinline__ int checked_page(const DecodeParams& p, int page) {
     if ((unsigned)page < (unsigned)p.num_pages) return page;
     set_status(p.status, KVS_ERR_INVALID_ARG);
@@ -106,12 +117,22 @@ decode_partial_kernel(DecodeParams p) {
     const size_t row_stride = (size_t)p.Hkv * D;             // elements between tokens of a page
     const size_t lane_off = (size_t)g * D + l16 * CH;
 
+    // the block-table entry of a block's token t0 + l16 is read one block ahead of its use
+    auto page_of = [&](int b) {
+        int e = 0, o;
+        if (b < nblocks) split_token(p, min(b * BLK + (l16 & (BLK - 1)), n - 1), e, o);
+        return (b < nblocks) ? bt[e] : 0;
+    };
+    int page_id = page_of(first);
     for (int b = first; b < nblocks; b += stride) {
         const int t0 = b * BLK;
         // row index (page * page_size + offset) of token t0 + l16, fetched once per block by every lane;
         // tokens past the end are clamped to the last one (their scores are discarded below)
         const int tl = min(t0 + (l16 & (BLK - 1)), n - 1);
-        const int my_row = checked_page(p, bt[tl / ps]) * ps + tl % ps;
+        int tl_entry, tl_off;
+        split_token(p, tl, tl_entry, tl_off);
+        const int my_row = checked_page(p, page_id) * ps + tl_off;
+        page_id = page_of(b + stride);
         // ---- all K rows of the block in flight, then the scores ----
         RowChunk<CH> raw[ROWS];
         int rowi[ROWS];
@@ -215,19 +236,32 @@ decode_partial_kernel(DecodeParams p) {
     }
 }
 
-// ---- tensor-core variant (head_dim 128, pages of 8..128 tokens) -----------------------------------
+// ---- tensor-core variant (head_dim 128) ------------------------------------------------------------
 // With G >= 4 query heads per KV head the CUDA-core kernel above is bound by its arithmetic (every K/V
 // element is multiplied G times in fp32), not by HBM.  Here the two products run on the tensor core in
 // the transposed form, so that the 128 keys of a tile (not the few query heads) fill the 128 rows:
 //   S^T [128 keys x 16] = K [128 x d] (Q_pad [16 x d])^T        A = K tile, B = Q (rows >= G are zero)
 //   O^T [d x 16]      += (V [128 keys x d])^T P^T [128 keys x 16]   A = V tile read MN-major, B = P^T
 // One CTA per (split, KV head, sequence), 4 softmax warps (thread = key in the S^T phase, = output
-// column d in the O^T phase) and one control warp (TMA loads of the tile's pages, MMA issue).  A tile
-// is processed serially; three CTAs per SM overlap one another's loads, MMAs and softmax.  Tensor
-// memory: 32 columns (S^T | O^T).  The per-head maximum over the 128 keys of a tile is a warp
+// column d in the O^T phase) and one control warp (block-table reads, TMA loads, MMA issue).  Three CTAs
+// per SM overlap one another's loads, MMAs and softmax.  Inside a CTA the K and the V buffer are
+// refilled at different times: K of tile t+1 is requested as soon as S^T of tile t is complete (the
+// softmax and the second product of tile t hide its latency), V of tile t as soon as the second product
+// of tile t-1 is complete (S^T and the softmax of tile t hide it).  How rows reach shared memory:
+//   pages of 8..128 tokens that tile 128 exactly: one TMA box per page and 64-column half;
+//   anything else (one token per page): K by TMA gather4, four cache rows per instruction, V by cp.async
+//   from the softmax warps, 16 lanes per 256-byte row.  A TMA instruction costs the SM's TMA unit about
+//   16 - 20 clocks whatever it moves, so with both K and V gathered (128 instructions per tile) the
+//   kernel is bound by that unit; splitting the rows between the TMA unit and the load/store unit is
+//   what gets past it.
+// Block-table entries are read with independent loads ahead of their use and checked afterwards: a load
+// whose value decides a branch at once would put one memory latency per entry into the tile's chain.
+// Tensor memory: 32 columns (S^T | O^T).  The per-head maximum over the 128 keys of a tile is a warp
 // reduction plus one exchange through shared memory; the reference maximum moves lazily (threshold
 // 8 in base-2 units), so O^T is rescaled in tensor memory only rarely.
 constexpr int DTC_THREADS = 160;
+constexpr int DTC_PAGES = 1;     // one TMA box per page
+constexpr int DTC_ROWS = 2;      // K: TMA gather4; V: cp.async rows
 
 struct DtcSmem {
     static constexpr int OFF_K = 0;                    // [128 keys x 128 d] bf16, two 64-column boxes, 128-byte swizzle
@@ -249,19 +283,29 @@ __device__ __forceinline__ int float_order(float x) {
 }
 __device__ __forceinline__ float float_unorder(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 
-template <int G, bool PAGED_TMA>
+// TMA gather: the 64-column slice starting at column c0 of the four rows r0..r3 of a 2-D tensor lands in four
+// consecutive 128-byte rows at dst (swizzled by address like a tiled box); completes 512 bytes on the barrier.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int c0, int r0, int r1, int r2, int r3, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
+        : "memory");
+}
+
+template <int G, int LOAD>
 __global__ void __launch_bounds__(DTC_THREADS, 3)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, DecodeParams p, int32_t* status) {
     constexpr int D = 128;
     constexpr int BOX = 16384;                  // one 64-column box of a 128-row tile
     constexpr uint32_t IDESC_S = make_idesc(16, 0, 0);
     constexpr uint32_t IDESC_O = make_idesc(16, 1, 0);
+    constexpr bool PAGES = LOAD == DTC_PAGES;
     extern __shared__ uint8_t smem_raw[];
     const int z = blockIdx.x, g = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n = min(max(p.n_tokens[s], 0), p.max_pages * p.page_size);    // never past the sequence's table
     const int ps = p.page_size;
-    const int ppt = 128 / ps;                                   // pages per tile
+    const int ppt = 128 / ps;                                   // pages per tile (PAGES)
     const int ntiles = (n + 127) >> 7;
     const int per = (ntiles + p.nsplit - 1) / p.nsplit;         // contiguous tiles per split
     const int t_begin = min(z * per, ntiles), t_end = min(t_begin + per, ntiles);
@@ -272,7 +316,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     uint8_t* sgen = smem_raw + (sbase - sraw);
     const uint32_t sK = sbase + DtcSmem::OFF_K, sV = sbase + DtcSmem::OFF_V, sQ = sbase + DtcSmem::OFF_Q, sP = sbase + DtcSmem::OFF_P;
     const uint32_t bars = sbase + DtcSmem::OFF_BAR;
-    const uint32_t bar_full = bars, bar_s = bars + 8, bar_p = bars + 16, bar_free = bars + 24;
+    // kfull / vfull: the tile's K / V rows have landed (TMA);  s: S^T is complete, hence K consumed and, the tensor pipe
+    // being in order, the previous tile's second product too (V, P^T consumed, O^T up to date);  p: P^T is written (and,
+    // with DTC_ROWS, the thread's V rows have landed);  done: the second product of a tile is complete
+    const uint32_t bar_kfull = bars, bar_vfull = bars + 8, bar_s = bars + 16, bar_p = bars + 24, bar_done = bars + 32;
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sgen + DtcSmem::OFF_MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + DtcSmem::OFF_MISC + 4);
     float* s_wmax = reinterpret_cast<float*>(sgen + DtcSmem::OFF_WMAX);
@@ -280,10 +327,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 
     if (tid == 0) {
         *abort_flag = 0;
-        mbar_init(bar_full, PAGED_TMA ? 1 : 128);
+        mbar_init(bar_kfull, 1);
+        mbar_init(bar_vfull, 1);
         mbar_init(bar_s, 1);
         mbar_init(bar_p, 128);
-        mbar_init(bar_free, 1);
+        mbar_init(bar_done, 1);
         fence_mbar_init();
     }
     if (warp == 4) {
@@ -309,30 +357,81 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     tc_fence_after();
     const uint32_t tmem = *s_tmem;
     const uint32_t tmem_S = tmem, tmem_O = tmem + 16;
+    const int32_t* bt = p.block_table + (size_t)s * p.max_pages;
 
     if (warp == 4) {
-        // ================= control warp: page loads and MMA issue =================
+        // ================= control warp: block table, TMA loads, MMA issue =================
         const bool leader = elect_one();
-        const int32_t* bt = p.block_table + (size_t)s * p.max_pages;
-        (void)bt;
         const uint64_t dK = smem_desc(sK, 16, 1024), dQ = smem_desc(sQ, 16, 1024);
         const uint64_t dV = smem_desc(sV, BOX, 1024), dP = smem_desc(sP, 16, 1024);
-        for (int it = 0; it < my_tiles; ++it) {
-            const int tt = t_begin + it;
-            const int npages = min(ppt, (n - tt * 128 + ps - 1) / ps);
-            if (PAGED_TMA && it > 0) mbar_wait(bar_free, (it - 1) & 1, abort_flag, status);     // K, V, P^T of the previous tile are consumed
-            if (PAGED_TMA && leader) {
-                mbar_expect_tx(bar_full, (uint32_t)(npages * ps) * 512u);
-                for (int i = 0; i < npages; ++i) {
-                    const int row = checked_page(p, bt[tt * ppt + i]) * ps;
-                    const uint32_t off = (uint32_t)(i * ps) * 128u;
-                    tma_load_3d(sK + off, &tm_k, 0, g, row, bar_full);
-                    tma_load_3d(sK + BOX + off, &tm_k, 64, g, row, bar_full);
-                    tma_load_3d(sV + off, &tm_v, 0, g, row, bar_full);
-                    tma_load_3d(sV + BOX + off, &tm_v, 64, g, row, bar_full);
+        // Block-table entries of a tile, held by the lanes: PAGES: lane i has page i of the tile (at most 16);
+        // ROWS: lane L has the pages of rows 4L .. 4L+3; a row past the end of the sequence repeats the last valid
+        // token (finite values, weight 0).
+        struct Ids { int v[PAGES ? 1 : 4]; };
+        auto fetch_ids = [&](int tt, Ids& id) {
+            if (tt >= t_end) return;
+            if (PAGES) {
+                const int npages = min(ppt, (n - tt * 128 + ps - 1) / ps);
+                id.v[0] = (lane < npages) ? bt[tt * ppt + lane] : 0;
+            } else {
+                const int nvalid = min(128, n - tt * 128);
+#pragma unroll
+                for (int j = 0; j < (PAGES ? 1 : 4); ++j) {
+                    int e, o;
+                    split_token(p, tt * 128 + min(4 * lane + j, nvalid - 1), e, o);
+                    id.v[j] = bt[e];
                 }
             }
-            mbar_wait(bar_full, it & 1, abort_flag, status);
+        };
+        auto load_k = [&](int tt, const Ids& id) {          // K buffer must be free
+            if (PAGES) {
+                const int npages = min(ppt, (n - tt * 128 + ps - 1) / ps);
+                const int row = checked_page(p, id.v[0]) * ps;
+                if (leader) mbar_expect_tx(bar_kfull, (uint32_t)(npages * ps) * 256u);
+                __syncwarp();
+                if (lane < npages) {
+                    const uint32_t off = (uint32_t)(lane * ps) * 128u;
+                    tma_load_3d(sK + off, &tm_k, 0, g, row, bar_kfull);
+                    tma_load_3d(sK + BOX + off, &tm_k, 64, g, row, bar_kfull);
+                }
+            } else {
+                const int nvalid = min(128, n - tt * 128);
+                const int ngroups = (nvalid + 3) >> 2;      // groups wholly past the end are not fetched
+                int row[4];
+#pragma unroll
+                for (int j = 0; j < (PAGES ? 1 : 4); ++j) {
+                    int e, o;
+                    split_token(p, tt * 128 + min(4 * lane + j, nvalid - 1), e, o);
+                    row[j] = checked_page(p, id.v[j]) * ps + o;
+                }
+                if (leader) mbar_expect_tx(bar_kfull, (uint32_t)ngroups * 1024u);
+                __syncwarp();
+                if (lane < ngroups) {
+                    const uint32_t off = (uint32_t)lane * 512u;
+                    tma_gather4(sK + off, &tm_k, g * D, row[0], row[1], row[2], row[3], bar_kfull);
+                    tma_gather4(sK + BOX + off, &tm_k, g * D + 64, row[0], row[1], row[2], row[3], bar_kfull);
+                }
+            }
+        };
+        auto load_v = [&](int tt, const Ids& id) {          // PAGES only; V buffer must be free
+            const int npages = min(ppt, (n - tt * 128 + ps - 1) / ps);
+            const int row = checked_page(p, id.v[0]) * ps;
+            if (leader) mbar_expect_tx(bar_vfull, (uint32_t)(npages * ps) * 256u);
+            __syncwarp();
+            if (lane < npages) {
+                const uint32_t off = (uint32_t)(lane * ps) * 128u;
+                tma_load_3d(sV + off, &tm_v, 0, g, row, bar_vfull);
+                tma_load_3d(sV + BOX + off, &tm_v, 64, g, row, bar_vfull);
+            }
+        };
+        Ids cur, nxt;
+        for (int j = 0; j < (PAGES ? 1 : 4); ++j) cur.v[j] = nxt.v[j] = 0;
+        fetch_ids(t_begin, cur);
+        fetch_ids(t_begin + 1, nxt);
+        if (my_tiles > 0) load_k(t_begin, cur);
+        for (int it = 0; it < my_tiles; ++it) {
+            const int tt = t_begin + it;
+            mbar_wait(bar_kfull, it & 1, abort_flag, status);
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {      // S^T = K Q^T, 16 elements of d per step
@@ -341,14 +440,20 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 if (leader) mma_ss(tmem_S, dK + offk, dQ + offq, IDESC_S, kk > 0);
             }
             if (leader) mma_commit(bar_s);
+            mbar_wait(bar_s, it & 1, abort_flag, status);      // K is consumed; so are V and P^T of the previous tile
+            if (PAGES) load_v(tt, cur);
+            if (it + 1 < my_tiles) load_k(tt + 1, nxt);
+            cur = nxt;
+            fetch_ids(tt + 2, nxt);
             mbar_wait(bar_p, it & 1, abort_flag, status);
+            if (PAGES) mbar_wait(bar_vfull, it & 1, abort_flag, status);
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {           // O^T += V^T P^T, 16 keys per step
                 const uint64_t offp = (uint64_t)(((kk >> 2) * 2048 + (kk & 3) * 32) >> 4);
                 if (leader) mma_ss(tmem_O, dV + (uint64_t)(kk * 128), dP + offp, IDESC_O, (it > 0) || (kk > 0));
             }
-            if (leader) mma_commit(bar_free);
+            if (leader) mma_commit(bar_done);
         }
     } else {
         // ================= softmax warps =================
@@ -359,60 +464,48 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             m_run[h] = -INFINITY;
             l_part[h] = 0.f;
         }
-        // Pages smaller than a swizzle atom (8 rows), e.g. one token per page: the softmax warps fetch the tile
-        // themselves, 16 lanes per 256-byte row (coalesced), with cp.async into the swizzled layout; rows past the
-        // end of the sequence are not fetched and keep their earlier, finite contents (their weight is 0).
-        const int32_t* bt = p.block_table + (size_t)s * p.max_pages;
-        // cache rows of this thread's 16 tokens of a tile (looked up one tile ahead, so that the block-table reads
-        // are not in the way when the tile's buffers become free); -1 = past the end of the sequence
-        long long nrow[16];
-        auto lookup_rows = [&](int tt) {
+        // DTC_ROWS: this thread's 16 rows of a tile's V (row r = warp * 32 + 2 j + lane / 16, 16 lanes per 256-byte row,
+        // cp.async into the swizzled layout).  Rows past the end of the sequence are not fetched and keep their earlier,
+        // finite contents (their weight is 0).  The block-table entries are loaded one tile ahead.
+        int pid[PAGES ? 1 : 16];
+        auto fetch_pids = [&](int tt) {
+            if (PAGES || tt >= t_end) return;
             const int nvalid = min(128, n - tt * 128);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int r = warp * 32 + 2 * j + (lane >> 4);
-                const int tok = tt * 128 + r;
-                nrow[j] = (r < nvalid) ? (long long)checked_page(p, bt[tok / ps]) * ps + tok % ps : -1;
+            for (int j = 0; j < (PAGES ? 1 : 16); ++j) {
+                int e, o;
+                split_token(p, tt * 128 + min(warp * 32 + 2 * j + (lane >> 4), nvalid - 1), e, o);
+                pid[j] = bt[e];
             }
         };
-        auto load_tile_rows = [&]() {
+        const __nv_bfloat16* v_lane = p.v_cache + (size_t)g * D + (lane & 15) * 8;       // this lane's 16 bytes of a row of head g
+        const int v_row_elems = p.Hkv * D;
+        auto load_v_rows = [&](int tt) {
+            const int nvalid = min(128, n - tt * 128);
             const int c = lane & 15;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
+            for (int j = 0; j < (PAGES ? 1 : 16); ++j) {
                 const int r = warp * 32 + 2 * j + (lane >> 4);
-                if (nrow[j] >= 0) {
-                    const size_t src = ((size_t)nrow[j] * p.Hkv + g) * D + c * 8;
+                int e, o;
+                split_token(p, tt * 128 + r, e, o);
+                const int crow = checked_page(p, pid[j]) * ps + o;
+                if (r < nvalid) {
                     const uint32_t dst = (uint32_t)((c >> 3) * BOX + r * 128 + (((c & 7) ^ (r & 7)) << 4));
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sK + dst), "l"(p.k_cache + src) : "memory");
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sV + dst), "l"(p.v_cache + src) : "memory");
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sV + dst), "l"(v_lane + (long long)crow * v_row_elems) : "memory");
                 }
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            fence_proxy_async();
-            mbar_arrive(bar_full);
         };
-        if (!PAGED_TMA && my_tiles > 0) {
-            lookup_rows(t_begin);
-            load_tile_rows();
-        }
+        fetch_pids(t_begin);
         for (int it = 0; it < my_tiles; ++it) {
             const int tt = t_begin + it;
-            if (!PAGED_TMA && it + 1 < my_tiles) lookup_rows(tt + 1);
             const int nvalid = min(128, n - tt * 128);
-            const int loaded = min(ppt, (n - tt * 128 + ps - 1) / ps) * ps;
-            mbar_wait(bar_full, it & 1, abort_flag, status);
-            if (PAGED_TMA && tid >= nvalid && tid < loaded) {
-                // rows of the last page past the end of the sequence were never written by anyone
-                const uint4 zero4 = make_uint4(0, 0, 0, 0);
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    *reinterpret_cast<uint4*>(sgen + DtcSmem::OFF_V + tid * 128 + c * 16) = zero4;
-                    *reinterpret_cast<uint4*>(sgen + DtcSmem::OFF_V + BOX + tid * 128 + c * 16) = zero4;
-                }
-            }
-            mbar_wait(bar_s, it & 1, abort_flag, status);
+            mbar_wait(bar_s, it & 1, abort_flag, status);       // S^T ready; V, P^T free; O^T up to date
             tc_fence_after();
+            if (!PAGES) {
+                load_v_rows(tt);
+                fetch_pids(tt + 1);
+            }
             uint32_t r[16];
             tmem_ld16(tmem_S + lane_sel, r);
             tmem_wait_ld();
@@ -464,17 +557,30 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 l_part[h] += w;
                 *reinterpret_cast<__nv_bfloat16*>(prow + h * 128 + ((chunk ^ (h & 7)) << 4)) = __float2bfloat16(w);
             }
-            fence_proxy_async();      // P^T (and the zeroed V rows) visible to the tensor core's reads of shared memory
+            if (PAGES) {
+                const int loaded = min(ppt, (n - tt * 128 + ps - 1) / ps) * ps;
+                if (loaded > nvalid) {            // the same decision in every thread
+                    // rows of the last page past the end of the sequence hold whatever the cache holds there
+                    mbar_wait(bar_vfull, it & 1, abort_flag, status);
+                    if (tid >= nvalid && tid < loaded) {
+                        const uint4 zero4 = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            *reinterpret_cast<uint4*>(sgen + DtcSmem::OFF_V + tid * 128 + c * 16) = zero4;
+                            *reinterpret_cast<uint4*>(sgen + DtcSmem::OFF_V + BOX + tid * 128 + c * 16) = zero4;
+                        }
+                    }
+                }
+            } else {
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+            }
+            fence_proxy_async();      // P^T and the V rows written by this thread visible to the tensor core's reads of shared memory
             tc_fence_before();
             mbar_arrive(bar_p);
-            if (!PAGED_TMA && it + 1 < my_tiles) {
-                mbar_wait(bar_free, it & 1, abort_flag, status);        // K, V of this tile are consumed
-                load_tile_rows();
-            }
         }
         // ---- this split's partial result: O^T (unnormalised), the reference maxima and the sums ----
         if (my_tiles > 0) {
-            mbar_wait(bar_free, (my_tiles - 1) & 1, abort_flag, status);
+            mbar_wait(bar_done, (my_tiles - 1) & 1, abort_flag, status);
             tc_fence_after();
         }
         uint32_t o[16];
@@ -739,14 +845,28 @@ extern "C" int kvs_cache_evict(const int32_t* ranges, int n_ranges, int num_seqs
 
 extern "C" int kvs_decode_num_splits(int num_seqs, int Hkv, int max_tokens) {
     if (num_seqs <= 0 || Hkv <= 0 || max_tokens <= 0) return 1;
-    // enough CTAs for two waves at three resident CTAs per SM (148 SMs), but at least 4 blocks of 16
-    // tokens per warp of a split
-    long long want = (2 * 3 * 148 + (long long)num_seqs * Hkv - 1) / ((long long)num_seqs * Hkv);
-    long long cap = ((long long)max_tokens + 16 * 4 * 4 - 1) / (16 * 4 * 4);
-    long long n = want < cap ? want : cap;
-    if (n < 1) n = 1;
-    if (n > 64) n = 64;
-    return (int)n;
+    // Three CTAs are resident per SM (148 SMs).  At least two waves of CTAs, at least 4 tiles of 128 tokens per split,
+    // and from there up to three times as many the first count whose last wave is at least 92 % full (else the
+    // fullest): a CTA of a sparse last wave runs at the latency of its own loads instead of sharing the memory
+    // system's bandwidth.
+    const long long slots = 3 * 148, base = (long long)num_seqs * Hkv;
+    long long want = (2 * slots + base - 1) / base;
+    long long cap = ((long long)max_tokens + 128 * 4 - 1) / (128 * 4);
+    if (cap > 64) cap = 64;
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    long long best = want;
+    double best_eff = 0.0;
+    for (long long n = want; n <= cap && n <= 3 * want; ++n) {
+        const long long ctas = base * n, waves = (ctas + slots - 1) / slots;
+        const double eff = (double)ctas / (double)(waves * slots);
+        if (eff > best_eff) {
+            best_eff = eff;
+            best = n;
+        }
+        if (eff >= 0.92) break;                 // the smallest count that fills its last wave well
+    }
+    return (int)best;
 }
 
 extern "C" size_t kvs_decode_workspace_bytes(int num_seqs, int Hq, int head_dim, int num_splits) {
@@ -761,9 +881,9 @@ __global__ void decode_header_kernel(int32_t* hdr) {
     hdr[1] = KVS_OK;
 }
 
-template <int G, bool PAGED_TMA>
+template <int G, int LOAD>
 static int launch_decode_tc(const CUtensorMap& tk, const CUtensorMap& tv, const DecodeParams& p, int32_t* status, cudaStream_t st) {
-    auto kern = decode_tc_kernel<G, PAGED_TMA>;
+    auto kern = decode_tc_kernel<G, LOAD>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DtcSmem::DYN_BYTES) != cudaSuccess) return KVS_ERR_CUDA;
     dim3 grid(p.nsplit, p.Hkv, p.S);
     kern<<<grid, DTC_THREADS, DtcSmem::DYN_BYTES, st>>>(tk, tv, p, status);
@@ -776,11 +896,11 @@ static int launch_decode(const DecodeParams& p, int G, const void* k_cache, cons
     dim3 grid(p.nsplit, p.Hkv, p.S);
     const int ps = p.page_size;
     // tensor-core variant (head_dim 128).  Pages that are whole 8-row swizzle atoms and tile 128 tokens exactly come in
-    // by TMA, one box per page: fastest for every group size.  Smaller pages (one token per page) come in by cp.async
-    // rows, which pays off from G = 4 on (measured: 0.56 of the HBM roofline against 0.70 for the CUDA-core kernel at
-    // G = 2, 0.50 against 0.28 at G = 7).
+    // by TMA, one box per page: at the HBM roofline for every group size.  Smaller pages (one token per page) come in
+    // row by row (K by TMA gather, V by cp.async), which beats the CUDA-core kernel from G = 2 on (measured at one
+    // token per page, fraction of the HBM roofline: G = 1 0.93 against 0.99, G = 2 0.93 against 0.84, G = 4 0.92).
     const bool paged_tma = (ps % 8 == 0) && (ps <= 128) && (128 % ps == 0);
-    const bool tc = (D == 128) && (G == 1 || G == 2 || G == 4 || G == 7 || G == 8) && (paged_tma || G >= 4);
+    const bool tc = (D == 128) && (G == 1 || G == 2 || G == 4 || G == 7 || G == 8) && (paged_tma || G >= 2);
     if (tc) {
         int rc = check_device_sm100();
         if (rc != KVS_OK) return rc;
@@ -794,19 +914,23 @@ static int launch_decode(const DecodeParams& p, int G, const void* k_cache, cons
             if ((rc = make_tmap_thd(&tk, k_cache, p.num_pages * ps, p.Hkv, 128, ps)) != KVS_OK) return rc;
             if ((rc = make_tmap_thd(&tv, v_cache, p.num_pages * ps, p.Hkv, 128, ps)) != KVS_OK) return rc;
             switch (G) {
-                case 1: rc = launch_decode_tc<1, true>(tk, tv, p, status, st); break;
-                case 2: rc = launch_decode_tc<2, true>(tk, tv, p, status, st); break;
-                case 4: rc = launch_decode_tc<4, true>(tk, tv, p, status, st); break;
-                case 7: rc = launch_decode_tc<7, true>(tk, tv, p, status, st); break;
-                default: rc = launch_decode_tc<8, true>(tk, tv, p, status, st); break;
+                case 1: rc = launch_decode_tc<1, DTC_PAGES>(tk, tv, p, status, st); break;
+                case 2: rc = launch_decode_tc<2, DTC_PAGES>(tk, tv, p, status, st); break;
+                case 4: rc = launch_decode_tc<4, DTC_PAGES>(tk, tv, p, status, st); break;
+                case 7: rc = launch_decode_tc<7, DTC_PAGES>(tk, tv, p, status, st); break;
+                default: rc = launch_decode_tc<8, DTC_PAGES>(tk, tv, p, status, st); break;
             }
         } else {
+            // the K cache as (Hkv * d, rows): a gather names four rows and a 64-column slice of one KV head (V is
+            // fetched with plain row copies and needs no tensor map)
+            if ((long long)p.num_pages * ps > 0x7fffffffLL) return KVS_ERR_UNSUPPORTED;
+            if ((rc = make_tmap_rows(&tk, k_cache, p.num_pages * ps, p.Hkv * 128)) != KVS_OK) return rc;
             switch (G) {
-                case 1: rc = launch_decode_tc<1, false>(tk, tv, p, status, st); break;
-                case 2: rc = launch_decode_tc<2, false>(tk, tv, p, status, st); break;
-                case 4: rc = launch_decode_tc<4, false>(tk, tv, p, status, st); break;
-                case 7: rc = launch_decode_tc<7, false>(tk, tv, p, status, st); break;
-                default: rc = launch_decode_tc<8, false>(tk, tv, p, status, st); break;
+                case 1: rc = launch_decode_tc<1, DTC_ROWS>(tk, tv, p, status, st); break;
+                case 2: rc = launch_decode_tc<2, DTC_ROWS>(tk, tv, p, status, st); break;
+                case 4: rc = launch_decode_tc<4, DTC_ROWS>(tk, tv, p, status, st); break;
+                case 7: rc = launch_decode_tc<7, DTC_ROWS>(tk, tv, p, status, st); break;
+                default: rc = launch_decode_tc<8, DTC_ROWS>(tk, tv, p, status, st); break;
             }
         }
         if (rc != KVS_OK) return rc;
@@ -848,6 +972,7 @@ extern "C" int kvs_decode_attn(const void* q, const void* k_cache, const void* v
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.page_size = page_size;
+    p.page_shift = (page_size & (page_size - 1)) == 0 ? __builtin_ctz((unsigned)page_size) : -1;
     p.max_pages = max_pages;
     p.num_pages = num_pages;
     p.status = (int32_t*)workspace + 1;

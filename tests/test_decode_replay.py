@@ -183,7 +183,8 @@ def test_batched_decode_three_sequences_and_error_reporting():
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("G,Hkv,ps", [(4, 2, 16), (8, 1, 16), (7, 2, 8), (8, 2, 32), (4, 1, 128), (8, 1, 64),
-                                      (8, 1, 1), (4, 2, 4), (7, 1, 3), (2, 2, 16), (1, 2, 1)])
+                                      (8, 1, 1), (4, 2, 4), (7, 1, 3), (2, 2, 16), (1, 2, 1), (2, 2, 1), (2, 1, 2), (4, 2, 1),
+                                      (1, 1, 5), (7, 2, 1)])
 def test_decode_attention_from_a_hand_built_cache(G, Hkv, ps):
     """Decode attention against its plain definition (softmax over exactly the rows the block table names), on a
     cache built by hand: scattered pages, lengths that end inside a page / inside a 128-token tile / at zero, and NaN

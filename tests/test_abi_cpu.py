@@ -52,6 +52,33 @@ def test_strerror_and_size_queries(lib):
     assert B.kvs_host_arena_bytes(1, 1024, 1024, 4, 4, 64, B.GRAD_BF16) > w16
 
 
+def test_host_arena_and_decode_split_sizing(lib):
+    from paper_2609_35750_b200 import binding as B
+    # the host entry point keeps three chunks of (trace range, KV head) on the device: with 8 KV heads a chunk is one head
+    # over all tokens, so the arena (three chunks with their fp32 dQ accumulators) is below the tensors; with one KV head the batch is cut into up to 8 trace ranges
+    T, d = 131072, 128
+    tensors = lambda Hq, Hkv: (2 * Hq + 2 * Hkv) * T * d * 2 * 2          # q, dout, out, dq + k, v, dk, dv in bf16
+    a8 = B.kvs_host_arena_bytes(2, T, 65536, 32, 8, d, B.GRAD_BF16)
+    assert 0 < a8 < 0.6 * tensors(32, 8)
+    a1_one = B.kvs_host_arena_bytes(1, T, T, 8, 1, d, B.GRAD_BF16)         # one trace cannot be cut
+    a1_many = B.kvs_host_arena_bytes(16, T, 8192, 8, 1, d, B.GRAD_BF16)    # 16 traces of 8192: 8 ranges of 2
+    assert a1_many < a1_one // 2
+    assert B.kvs_host_arena_bytes(2, T, 65536, 32, 5, d, B.GRAD_BF16) == 0      # Hq % Hkv != 0
+    assert B.kvs_host_arena_bytes(0, 0, 0, 32, 8, d, B.GRAD_BF16) == 256
+    # split count of decode attention: at least one, never more than a split per 4 tiles of 128 tokens, and the last wave
+    # of three CTAs per SM is at least 92 % full whenever some count in range allows it
+    slots = 3 * 148
+    for S, Hkv, n in [(32, 8, 12288), (64, 4, 7168), (16, 8, 16384), (8, 8, 32768), (256, 8, 2048), (1, 8, 100000), (1, 1, 300), (4, 2, 4096)]:
+        k = lib.kvs_decode_num_splits(S, Hkv, n)
+        cap = min(64, (n + 511) // 512)
+        assert 1 <= k <= max(cap, 1), (S, Hkv, n, k)
+        want = max(1, min(cap, -(-2 * slots // (S * Hkv))))
+        eff = lambda m: S * Hkv * m / (-(-S * Hkv * m // slots) * slots)
+        best = max(eff(m) for m in range(want, min(cap, 3 * want) + 1))
+        assert eff(k) >= min(0.92, best) - 1e-9, (S, Hkv, n, k, eff(k), best)
+    assert lib.kvs_decode_num_splits(0, 8, 100) == 1 and lib.kvs_decode_num_splits(4, 8, 0) == 1
+
+
 def test_host_side_argument_errors_need_no_gpu(lib):
     from paper_2609_35750_b200 import binding as B
     # null pointers / bad dims are rejected before any CUDA call

@@ -236,3 +236,58 @@ def test_decode_attention_from_a_hand_built_cache(G, Hkv, ps):
                 ref_o, ref_l = (w[:, None] * vv[:, h // G]).sum(0) / w.sum(), mx + np.log(w.sum())
                 assert np.isfinite(out[s, h]).all(), (s, h, n)
                 assert np.abs(out[s, h] - ref_o).max() < 2e-2 and abs(lse[s, h] - ref_l) < 2e-3, (splits, s, h, n)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", range(12))
+def test_decode_attention_fuzz(seed):
+    """Seeded random shapes of the decode step against its plain definition: page size, group width, KV heads, head
+    dimension, number of sequences, lengths (zero, one, ragged, several tiles), scattered pages with NaN in every row
+    that holds no token, split count chosen by the library or forced."""
+    from paper_2609_35750_b200 import binding as B
+    rng = np.random.default_rng(9000 + seed)
+    d = 64 if seed % 6 == 5 else 128
+    ps = int(rng.choice([1, 1, 2, 3, 4, 8, 16, 16, 32, 64, 128]))
+    G = int(rng.choice([1, 2, 4, 7, 8]))
+    Hkv = int(rng.choice([1, 2, 3]))
+    Hq = G * Hkv
+    S = int(rng.integers(1, 7))
+    lens = [int(x) for x in rng.choice([0, 1, ps, 127, 128, 129, 255, 640, 1500, 2900], size=S)]
+    lens[int(rng.integers(0, S))] = int(rng.integers(1, 3000))
+    max_pages = (max(lens) + ps - 1) // ps + 2
+    num_pages = sum((n + ps - 1) // ps for n in lens) + 3
+    k_cache = torch.full((num_pages, ps, Hkv, d), float("nan"), dtype=torch.bfloat16)
+    v_cache = torch.full((num_pages, ps, Hkv, d), float("nan"), dtype=torch.bfloat16)
+    table = torch.zeros((S, max_pages), dtype=torch.int32)
+    perm, nxt, rows = rng.permutation(num_pages), 0, []
+    for s, n in enumerate(lens):
+        kk = torch.from_numpy(rng.standard_normal((n, Hkv, d)).astype(np.float32)).to(torch.bfloat16)
+        vv = torch.from_numpy(rng.standard_normal((n, Hkv, d)).astype(np.float32)).to(torch.bfloat16)
+        rows.append((kk, vv))
+        for pi in range((n + ps - 1) // ps):
+            page = int(perm[nxt]); nxt += 1
+            table[s, pi] = page
+            m = min(ps, n - pi * ps)
+            k_cache[page, :m] = kk[pi * ps: pi * ps + m]
+            v_cache[page, :m] = vv[pi * ps: pi * ps + m]
+    q = torch.from_numpy((rng.standard_normal((S, Hq, d)) * rng.choice([0.5, 1.0, 3.0])).astype(np.float32)).to(torch.bfloat16)
+    cache = B.PagedCache(num_pages, ps, S, max_pages, Hkv, d)
+    cache.k_cache.copy_(k_cache)
+    cache.v_cache.copy_(v_cache)
+    cache.block_table.copy_(table)
+    cache.n_tokens.copy_(torch.tensor(lens, dtype=torch.int32))
+    splits = int(rng.choice([0, 0, 1, 2, 5]))
+    out, lse = cache.decode(q.cuda(), num_splits=splits, max_tokens=max(max(lens), 1))
+    out, lse = out.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+    scale = 1.0 / np.sqrt(d)
+    for s, n in enumerate(lens):
+        kk, vv = (t.float().numpy().astype(np.float64) for t in rows[s])
+        for h in range(Hq):
+            if n == 0:
+                assert np.all(out[s, h] == 0) and lse[s, h] == -np.inf
+                continue
+            sc = kk[:, h // G] @ q[s, h].float().numpy().astype(np.float64) * scale
+            w = np.exp(sc - sc.max())
+            ref_o, ref_l = (w[:, None] * vv[:, h // G]).sum(0) / w.sum(), sc.max() + np.log(w.sum())
+            assert np.isfinite(out[s, h]).all(), (ps, G, s, h, n)
+            assert np.abs(out[s, h] - ref_o).max() < 2e-2 and abs(lse[s, h] - ref_l) < 2e-3, (ps, G, Hkv, d, splits, s, h, n)

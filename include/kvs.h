@@ -300,6 +300,16 @@ size_t kvs_host_arena_bytes(int batch, int total_tokens, int max_seqlen,
                             int Hq, int Hkv, int head_dim, int grad_dtype);
 
 /*
+ * How kvs_attn_fwd_bwd_host cuts a batch into ranges of traces (host arrays only, no CUDA call): range i covers
+ * traces [range_traces[2 i], range_traces[2 i + 1]).  range_traces: host int32, room for 2 * batch entries.
+ * The ranges are contiguous, in order, leave out only traces without tokens, are at most ceil(8 / Hkv) (and at most
+ * batch), and none holds more than total_tokens / ranges + max_seqlen tokens.  Returns KVS_ERR_INVALID_ARG for a
+ * malformed cu_seqlens.
+ */
+int kvs_host_chunk_plan(const int32_t* cu_seqlens_host, int batch, int total_tokens, int max_seqlen, int Hkv,
+                        int32_t* range_traces, int* num_ranges);
+
+/*
  * Whole path from HOST buffers (the call a trainer without device tensors makes): copies
  * evict_at, cu_seqlens, q, k, v, dout to the device arena, runs mask metadata, forward and
  * backward, copies out, lse, dq, dk, dv back, and SYNCHRONISES the stream.  Host buffers

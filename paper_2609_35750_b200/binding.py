@@ -59,6 +59,7 @@ SIGNATURES = {
     "kvs_cache_append": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvs_cache_evict": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "kvs_cache_status": (_i, [_vp, ctypes.POINTER(ctypes.c_int), _vp]),
+    "kvs_host_chunk_plan": (_i, [_vp, _i, _i, _i, _i, _vp, ctypes.POINTER(ctypes.c_int)]),
     "kvs_decode_num_splits": (_i, [_i, _i, _i]),
     "kvs_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "kvs_decode_attn": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _sz, _vp]),
@@ -310,6 +311,19 @@ def kvs_rope_qk(q, k, cu_seqlens=None, positions=None, theta_base: float = 10000
                               q.shape[1] if q is not None else 0, k.shape[1] if k is not None else 0, d, float(theta_base), dt,
                               1 if inverse else 0, ptr(q_out, "q_out"), ptr(k_out, "k_out"), _stream(stream)), "kvs_rope_qk")
     return q_out, k_out
+
+
+def kvs_host_chunk_plan(cu_seqlens, max_seqlen: int, Hkv: int):
+    """The trace ranges kvs_attn_fwd_bwd_host cuts a batch into: a list of (first trace, one past the last).
+    cu_seqlens: int32 numpy array or CPU tensor [batch + 1].  Host only."""
+    import numpy as np
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens), dtype=np.int32)
+    batch = int(cu.shape[0]) - 1
+    buf = np.zeros(max(2 * batch, 2), dtype=np.int32)
+    n = ctypes.c_int(0)
+    _check(load().kvs_host_chunk_plan(cu.ctypes.data, batch, int(cu[-1]) if batch >= 0 else 0, int(max_seqlen), int(Hkv), buf.ctypes.data,
+                                      ctypes.byref(n)), "kvs_host_chunk_plan")
+    return [(int(buf[2 * i]), int(buf[2 * i + 1])) for i in range(n.value)]
 
 
 def kvs_attn_bwd_workspace_bytes(total_tokens: int, Hq: int, Hkv: int, head_dim: int, grad_dtype: int) -> int:

@@ -175,6 +175,41 @@ inline int host_ranges(int batch, int Hkv) {
     return r < 1 ? 1 : r;
 }
 
+// A contiguous range of traces [b0, b1): its first token, token count, longest trace, and where its re-based
+// cu_seqlens (b1 - b0 + 1 entries starting with 0) sit in the staging array.
+struct Range { int b0, b1, tok0, tokens, maxlen, cu_off; };
+
+// Cuts the batch into at most `want` contiguous ranges of traces: a range is closed once it holds its share
+// ceil(total / want) of the tokens (so it exceeds the share by less than one trace) or when the traces left are
+// only enough to give every remaining range one; the last range takes what is left.  Ranges without a token are dropped.
+void plan_trace_ranges(const int32_t* cu, int batch, int total_tokens, int want, std::vector<Range>& ranges, std::vector<int32_t>& cu_ranges) {
+    ranges.clear();
+    cu_ranges.clear();
+    if (want < 1) want = 1;
+    const long long share = ((long long)total_tokens + want - 1) / want;
+    int b = 0;
+    while (b < batch) {
+        Range r;
+        r.b0 = b;
+        r.tok0 = cu[b];
+        r.maxlen = 0;
+        r.cu_off = (int)cu_ranges.size();
+        cu_ranges.push_back(0);
+        const int left_ranges = want - (int)ranges.size();          // >= 1: the last one takes all that is left
+        while (b < batch) {
+            const int T = cu[b + 1] - cu[b];
+            cu_ranges.push_back(cu[b + 1] - r.tok0);
+            if (T > r.maxlen) r.maxlen = T;
+            ++b;
+            if (left_ranges > 1 && ((long long)cu[b] - r.tok0 >= share || batch - b <= left_ranges - 1)) break;
+        }
+        r.b1 = b;
+        r.tokens = cu[b] - r.tok0;
+        if (r.tokens > 0) ranges.push_back(r);
+        else cu_ranges.resize(r.cu_off);
+    }
+}
+
 struct ArenaLayout {
     size_t evict, cu, sticky, meta, slot0, slot_stride, total;      // global part, then HOST_SLOTS equal slots
     size_t q, k, v, dout, out, lse, dq, dk, dv, ws;                  // offsets inside a slot
@@ -228,6 +263,27 @@ extern "C" size_t kvs_host_arena_bytes(int batch, int total_tokens, int max_seql
     return arena_layout(batch, total_tokens, max_seqlen, Hq, Hkv, head_dim, grad_dtype).total;
 }
 
+extern "C" int kvs_host_chunk_plan(const int32_t* cu_seqlens_host, int batch, int total_tokens, int max_seqlen, int Hkv,
+                                   int32_t* range_trace_begin, int* num_ranges) {
+    if (!cu_seqlens_host || !range_trace_begin || !num_ranges || batch < 0 || total_tokens < 0 || Hkv <= 0) return KVS_ERR_INVALID_ARG;
+    *num_ranges = 0;
+    if (batch == 0 || total_tokens == 0) return KVS_OK;
+    if (cu_seqlens_host[0] != 0 || cu_seqlens_host[batch] != total_tokens) return KVS_ERR_INVALID_ARG;
+    for (int b = 0; b < batch; ++b) {
+        const long long T = (long long)cu_seqlens_host[b + 1] - cu_seqlens_host[b];
+        if (T < 0 || T > max_seqlen) return KVS_ERR_INVALID_ARG;
+    }
+    std::vector<Range> ranges;
+    std::vector<int32_t> cu_ranges;
+    plan_trace_ranges(cu_seqlens_host, batch, total_tokens, host_ranges(batch, Hkv), ranges, cu_ranges);
+    for (size_t i = 0; i < ranges.size(); ++i) {
+        range_trace_begin[2 * i] = ranges[i].b0;
+        range_trace_begin[2 * i + 1] = ranges[i].b1;
+    }
+    *num_ranges = (int)ranges.size();
+    return KVS_OK;
+}
+
 extern "C" int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t* cu_seqlens_host, const void* q_host,
                                      const void* k_host, const void* v_host, const void* dout_host, int batch, int total_tokens,
                                      int max_seqlen, int Hq, int Hkv, int head_dim, float softmax_scale, int grad_dtype,
@@ -265,35 +321,8 @@ extern "C" int kvs_attn_fwd_bwd_host(const int32_t* evict_at_host, const int32_t
     if (!R.in && cudaStreamCreateWithFlags(&R.in, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
     if (!R.outs && cudaStreamCreateWithFlags(&R.outs, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
 
-    // trace ranges: contiguous, each closed once it holds its share of the tokens
-    struct Range { int b0, b1, tok0, tokens, maxlen, cu_off; };
     std::vector<Range> ranges;
-    R.cu_ranges.clear();
-    {
-        const long long share = ((long long)total_tokens + A.ranges - 1) / A.ranges;
-        int b = 0;
-        while (b < batch) {
-            Range r;
-            r.b0 = b;
-            r.tok0 = cu_seqlens_host[b];
-            r.maxlen = 0;
-            r.cu_off = (int)R.cu_ranges.size();
-            R.cu_ranges.push_back(0);
-            const int left_ranges = A.ranges - (int)ranges.size();      // >= 1: the last one takes all that is left
-            while (b < batch) {
-                const int T = cu_seqlens_host[b + 1] - cu_seqlens_host[b];
-                R.cu_ranges.push_back(cu_seqlens_host[b + 1] - r.tok0);
-                if (T > r.maxlen) r.maxlen = T;
-                ++b;
-                const bool last_range = left_ranges <= 1;
-                if (!last_range && ((long long)cu_seqlens_host[b] - r.tok0 >= share || batch - b <= left_ranges - 1)) break;
-            }
-            r.b1 = b;
-            r.tokens = cu_seqlens_host[b] - r.tok0;
-            if (r.tokens > 0) ranges.push_back(r);          // a range of empty traces has no rows to compute or copy
-            else R.cu_ranges.resize(r.cu_off);
-        }
-    }
+    plan_trace_ranges(cu_seqlens_host, batch, total_tokens, A.ranges, ranges, R.cu_ranges);
     const int NR = (int)ranges.size();
     for (const Range& r : ranges)
         if (r.tokens > A.slot_tokens) return KVS_ERR_WORKSPACE;      // cannot happen: see arena_layout

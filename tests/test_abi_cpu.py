@@ -79,6 +79,51 @@ def test_host_arena_and_decode_split_sizing(lib):
     assert lib.kvs_decode_num_splits(0, 8, 100) == 1 and lib.kvs_decode_num_splits(4, 8, 0) == 1
 
 
+def test_host_chunk_plan_properties(lib):
+    """The trace ranges of the host-buffer entry point, on seeded random batches: contiguous and in order, every trace
+    with tokens covered exactly once, no range without tokens, at most min(batch, ceil(8 / Hkv)) ranges, none larger
+    than the slot the arena provides (total / ranges + the longest trace)."""
+    import numpy as np
+    from paper_2609_35750_b200 import binding as B
+    rng = np.random.default_rng(77)
+    for case in range(300):
+        batch = int(rng.integers(1, 40))
+        Hkv = int(rng.choice([1, 2, 3, 4, 8, 16]))
+        kind = case % 4
+        if kind == 0:
+            lens = rng.integers(0, 5000, size=batch)
+        elif kind == 1:
+            lens = np.where(rng.random(batch) < 0.4, 0, rng.integers(1, 300, size=batch))      # many empty traces
+        elif kind == 2:
+            lens = rng.integers(1, 50, size=batch); lens[int(rng.integers(0, batch))] = 100000     # one giant trace
+        else:
+            lens = np.full(batch, int(rng.integers(1, 4096)))
+        if lens.sum() == 0:
+            lens[0] = 1
+        cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        total, maxlen = int(cu[-1]), int(lens.max())
+        plan = B.kvs_host_chunk_plan(cu, maxlen, Hkv)
+        want = max(1, min(batch, -(-8 // Hkv)))
+        assert 1 <= len(plan) <= want, (case, plan)
+        covered = np.zeros(batch, dtype=bool)
+        prev_end = 0
+        for b0, b1 in plan:
+            assert prev_end <= b0 < b1 <= batch
+            assert lens[prev_end:b0].sum() == 0                       # only empty traces are skipped
+            tokens = int(cu[b1] - cu[b0])
+            assert 0 < tokens <= total // want + maxlen
+            covered[b0:b1] = True
+            prev_end = b1
+        assert lens[prev_end:].sum() == 0 and lens[~covered].sum() == 0
+    # malformed tables are refused
+    with pytest.raises(B.KvsError):
+        B.kvs_host_chunk_plan(np.array([0, 5, 3], dtype=np.int32), 10, 1)
+    with pytest.raises(B.KvsError):
+        B.kvs_host_chunk_plan(np.array([1, 5, 8], dtype=np.int32), 10, 1)
+    with pytest.raises(B.KvsError):
+        B.kvs_host_chunk_plan(np.array([0, 50, 80], dtype=np.int32), 10, 1)         # a trace longer than max_seqlen
+
+
 def test_host_side_argument_errors_need_no_gpu(lib):
     from paper_2609_35750_b200 import binding as B
     # null pointers / bad dims are rejected before any CUDA call

@@ -370,6 +370,59 @@ def test_host_buffer_entry_point_reports_bad_masks_and_bad_trace_tables():
     assert torch.equal(good[0], out.cpu()) and torch.equal(good[1], lse.cpu()) and torch.equal(good[3], dk.cpu())
 
 
+def test_whole_step_replays_from_a_cuda_graph():
+    # mask metadata + forward + backward allocate nothing and never synchronise, so a step can be captured once and
+    # replayed: new masks and tensors written into the captured buffers give the new step's results, equal to the
+    # eager calls (dq within its reduction-order noise), at a fraction of the launch cost on a small batch
+    w1 = W.make_workload(2, seed=11, shrink=64, Hq=8, Hkv=2, batch=2)
+    w2 = W.make_workload(2, seed=12, shrink=64, Hq=8, Hkv=2, batch=2)          # same sizes, other turn lengths and evictions
+    assert w1.total_tokens == w2.total_tokens and w1.max_seqlen == w2.max_seqlen
+    grad = B.GRAD_BF16
+    ev = torch.from_numpy(w1.evict_at).to(DEV)
+    cu = torch.from_numpy(w1.cu_seqlens).to(DEV)
+    q, k, v, do = (t.to(DEV) for t in W.make_tensors(w1, 1))
+    meta = torch.empty(B.kvs_mask_meta_bytes(w1.batch, w1.total_tokens, w1.max_seqlen), dtype=torch.uint8, device=DEV)
+    ws = torch.empty(B.kvs_attn_bwd_workspace_bytes(w1.total_tokens, w1.Hq, w1.Hkv, w1.d, grad), dtype=torch.uint8, device=DEV)
+    out, lse = torch.empty_like(q), torch.empty((w1.Hq, w1.total_tokens), dtype=torch.float32, device=DEV)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+
+    def step():
+        B.kvs_mask_meta(ev, cu, w1.max_seqlen, meta_buf=meta)
+        B.kvs_attn_fwd(q, k, v, meta, w1.batch, w1.max_seqlen, w1.softmax_scale, out=out, lse=lse)
+        B.kvs_attn_bwd(do, q, k, v, out, lse, meta, w1.batch, w1.max_seqlen, w1.softmax_scale, grad, dq=dq, dk=dk, dv=dv, workspace=ws)
+
+    step()                                                   # eager once: function attributes and modules are set up
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    for w, seed in ((w2, 2), (w1, 1)):
+        tq, tk, tv, tdo = (t.to(DEV) for t in W.make_tensors(w, seed))
+        ev.copy_(torch.from_numpy(w.evict_at)); cu.copy_(torch.from_numpy(w.cu_seqlens))
+        q.copy_(tq); k.copy_(tk); v.copy_(tv); do.copy_(tdo)
+        for t in (out, dq, dk, dv):
+            t.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert B.kvs_device_status(meta) == B.KVS_OK and B.kvs_device_status(ws) == B.KVS_OK
+        _, ro, rl, rdq, rdk, rdv = _run_gpu(w, tq, tk, tv, tdo, grad)
+        assert torch.equal(out, ro) and torch.equal(lse, rl) and torch.equal(dk, rdk) and torch.equal(dv, rdv)
+        assert torch.allclose(dq.float(), rdq.float(), atol=2e-2, rtol=2e-2)
+    # launch cost: 20 replays against 20 eager steps on this small batch
+    a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    a.record()
+    for _ in range(20):
+        step()
+    b.record()
+    for _ in range(20):
+        graph.replay()
+    c.record()
+    torch.cuda.synchronize()
+    print(f"eager {a.elapsed_time(b) / 20:.3f} ms per step, graph replay {b.elapsed_time(c) / 20:.3f} ms per step")
+
+
 # ---- the error of the CUDA path is the method's own operand rounding -------------------------------
 @pytest.mark.parametrize("kw", [dict(cfg=0), dict(cfg=2, shrink=32, Hq=8, Hkv=2, batch=1), dict(cfg=4, shrink=64, Hq=8, Hkv=1)])
 def test_error_is_explained_by_the_operand_rounding_model(kw):

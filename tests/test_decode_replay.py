@@ -291,3 +291,67 @@ def test_decode_attention_fuzz(seed):
             ref_o, ref_l = (w[:, None] * vv[:, h // G]).sum(0) / w.sum(), sc.max() + np.log(w.sum())
             assert np.isfinite(out[s, h]).all(), (ps, G, s, h, n)
             assert np.abs(out[s, h] - ref_o).max() < 2e-2 and abs(lse[s, h] - ref_l) < 2e-3, (ps, G, Hkv, d, splits, s, h, n)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("ps", [16, 1])
+def test_decode_step_replays_from_a_cuda_graph(ps):
+    """Appending a token and attending over the live cache keep their state (token counts, block tables, free stack)
+    on the device and take no host decision, so the pair can be captured once and replayed for every generated token,
+    as rollout engines do; the results equal the eager calls token by token."""
+    from paper_2609_35750_b200 import binding as B
+    rng = np.random.default_rng(5 + ps)
+    S, Hkv, G, d, T = 3, 2, 4, 128, 200
+    Hq = G * Hkv
+    num_pages, max_pages = S * ((T + ps - 1) // ps) + 2, (T + ps - 1) // ps + 1
+    ks = torch.from_numpy(rng.standard_normal((T, S, Hkv, d)).astype(np.float32)).to(torch.bfloat16).cuda()
+    vs = torch.from_numpy(rng.standard_normal((T, S, Hkv, d)).astype(np.float32)).to(torch.bfloat16).cuda()
+    qs = torch.from_numpy(rng.standard_normal((T, S, Hq, d)).astype(np.float32)).to(torch.bfloat16).cuda()
+    splits = 2
+
+    def run(graphed):
+        cache = B.PagedCache(num_pages, ps, S, max_pages, Hkv, d)
+        q, k, v = torch.empty_like(qs[0]), torch.empty_like(ks[0]), torch.empty_like(vs[0])
+        out, lse = torch.empty_like(q), torch.empty((S, Hq), dtype=torch.float32, device="cuda")
+        ws = torch.empty(int(B.load().kvs_decode_workspace_bytes(S, Hq, d, splits)), dtype=torch.uint8, device="cuda")
+        outs, lses = [], []
+
+        def step():
+            cache.append(k, v)
+            cache.decode(q, num_splits=splits, out=out, lse=lse, workspace=ws)
+
+        graph, first = None, 0
+        if graphed:
+            q.copy_(qs[0]); k.copy_(ks[0]); v.copy_(vs[0])
+            step()                                      # token 0 eagerly (sets up function attributes), then capture
+            outs.append(out.clone()); lses.append(lse.clone())
+            first = 1
+            torch.cuda.synchronize()
+            graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(graph, stream=side):
+                    step()
+            # the capture itself ran nothing: the cache still holds one token per sequence
+            assert cache.n_tokens.cpu().tolist() == [1] * S
+        for i in range(first, T):
+            q.copy_(qs[i]); k.copy_(ks[i]); v.copy_(vs[i])
+            if graphed:
+                graph.replay()
+            else:
+                step()
+            outs.append(out.clone()); lses.append(lse.clone())
+        torch.cuda.synchronize()
+        assert cache.status()[0] == B.KVS_OK and cache.n_tokens.cpu().tolist() == [T] * S
+        return torch.stack(outs), torch.stack(lses)
+
+    eo, el = run(False)
+    go, gl = run(True)
+    assert torch.equal(eo, go) and torch.equal(el, gl)
+    # and the eager path is the definition: the last token against a plain softmax over all T keys
+    kk, vv, qq = (t.float().cpu().numpy().astype(np.float64) for t in (ks, vs, qs))
+    for s in range(S):
+        for h in range(Hq):
+            sc = kk[:, s, h // G] @ qq[T - 1, s, h] / np.sqrt(d)
+            w = np.exp(sc - sc.max())
+            ref = (w[:, None] * vv[:, s, h // G]).sum(0) / w.sum()
+            assert np.abs(eo[T - 1, s, h].float().cpu().numpy() - ref).max() < 2e-2

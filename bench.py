@@ -360,54 +360,58 @@ def run_meta_only(args):
         raise SystemExit(1)
 
 
-def run_decode(args):
-    """--path decode: one step = kvs_decode_attn for one new token of every sequence over its live cache.  The kernel
-    reads every live K and V row once, so it is bound by HBM: algorithmic bytes = live K and V rows of the sequences'
-    KV heads.  The block tables point at randomly permuted pages, the state of a cache after many evictions."""
+def measure_decode(hq, hkv, S, n, ps, head_dim=128, splits=0, steps=50, warmup=3):
+    """One step = kvs_decode_attn for one new token of every sequence over its live cache.  The kernel reads every live
+    K and V row once, so it is bound by HBM: algorithmic bytes = live K and V rows of the sequences' KV heads.  The block
+    tables point at randomly permuted pages, the state of a cache after many evictions."""
     import torch
     from paper_2609_35750_b200 import binding as B
     dev = "cuda"
-    hq, hkv = args.hq or 28, args.hkv or 4
-    S, n, ps = args.seqs, args.live, args.page_size
     pages_per_seq = (n + ps - 1) // ps
     num_pages = S * pages_per_seq + 8
-    cache = B.PagedCache(num_pages, ps, S, pages_per_seq, hkv, args.head_dim, device=dev)
+    cache = B.PagedCache(num_pages, ps, S, pages_per_seq, hkv, head_dim, device=dev)
     g = torch.Generator(device=dev).manual_seed(0)
     cache.k_cache.copy_(torch.randn(cache.k_cache.shape, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16))
     cache.v_cache.copy_(torch.randn(cache.v_cache.shape, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16))
     perm = torch.randperm(num_pages, generator=g, device=dev)[: S * pages_per_seq].to(torch.int32)
     cache.block_table.copy_(perm.view(S, pages_per_seq))
     cache.n_tokens.fill_(n)
-    q = torch.randn((S, hq, args.head_dim), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
-    splits = args.splits or int(B.load().kvs_decode_num_splits(S, hkv, n))
-    ws = torch.empty(int(B.load().kvs_decode_workspace_bytes(S, hq, args.head_dim, splits)), dtype=torch.uint8, device=dev)
+    q = torch.randn((S, hq, head_dim), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    splits = splits or int(B.load().kvs_decode_num_splits(S, hkv, n))
+    ws = torch.empty(int(B.load().kvs_decode_workspace_bytes(S, hq, head_dim, splits)), dtype=torch.uint8, device=dev)
     out = torch.empty_like(q)
     lse = torch.empty((S, hq), dtype=torch.float32, device=dev)
-    for _ in range(max(args.warmup, 1)):
+    for _ in range(max(warmup, 1)):
         cache.decode(q, num_splits=splits, out=out, lse=lse, workspace=ws)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(args.steps):
+    for _ in range(steps):
         cache.decode(q, num_splits=splits, out=out, lse=lse, workspace=ws)
     e1.record()
     torch.cuda.synchronize()
     if B.kvs_device_status(ws) != 0:
         raise SystemExit("device status after the timed region: %d" % B.kvs_device_status(ws))
-    ms = e0.elapsed_time(e1) / args.steps
-    algo = 2.0 * S * n * hkv * args.head_dim * 2          # K and V rows, bf16
+    ms = e0.elapsed_time(e1) / steps
+    algo = 2.0 * S * n * hkv * head_dim * 2          # K and V rows, bf16
     peaks = load_peaks()
     gbs = algo / (ms * 1e-3) / 1e9
-    print(json.dumps({
-        "metric": "decode_attn_hbm_gbs", "value": gbs, "unit": "GB/s", "ms_per_step": ms, "steps": args.steps, "warmup": args.warmup,
+    return {
+        "metric": "decode_attn_hbm_gbs", "value": gbs, "unit": "GB/s", "ms_per_step": ms, "steps": steps, "warmup": warmup,
         "config": {"workload": "decode over a fragmented paged cache", "seqs": S, "live_tokens": n, "page_size": ps, "Hq": hq,
-                   "Hkv": hkv, "head_dim": args.head_dim, "splits": splits,
+                   "Hkv": hkv, "head_dim": head_dim, "splits": splits,
                    "l2": "K/V working set %.0f MB, larger than L2" % (algo / 1e6)},
         "tokens_per_s": S / (ms * 1e-3),
         "roofline": {"kernel": "decode attention (partial + combine)", "bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]),
                      "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]), "traffic": None,
                      "peak_source": peaks["_source"] + " copy bandwidth"},
-        "dtype": "bf16", "data": "synthetic"}), flush=True)
+        "dtype": "bf16", "data": "synthetic"}
+
+
+def run_decode(args):
+    """--path decode: the rollout-side decode step on one shape, one JSON line."""
+    print(json.dumps(measure_decode(args.hq or 28, args.hkv or 4, args.seqs, args.live, args.page_size, args.head_dim, args.splits,
+                                    args.steps, args.warmup)), flush=True)
 
 
 def run_dual(args):
@@ -620,8 +624,17 @@ def main():
 
     peaks = load_peaks()
     per_config = None
+    rollout_decode = None
     if world == 1 and not small and args.config == 2 and args.variant == "" and not args.no_per_config:
         per_config = run_per_config(torch, B, W, dev, peaks, local_rank)
+        # the rollout side on the same clock: one decode step over config 1's peak cache and over a wider one,
+        # with 16-token and 1-token pages (fraction of the measured HBM copy bandwidth)
+        rollout_decode = {}
+        for name, (hq_, hkv_, S_, n_) in (("64x7168_Hq28_Hkv4", (28, 4, 64, 7168)), ("32x12288_Hq32_Hkv8", (32, 8, 32, 12288))):
+            for ps_ in (16, 1):
+                r = measure_decode(hq_, hkv_, S_, n_, ps_, steps=30, warmup=3)
+                rollout_decode[f"{name}_pages{ps_}"] = {"ms_per_step": r["ms_per_step"], "gbs": r["value"], "frac_of_hbm": r["roofline"]["frac"],
+                                                        "splits": r["config"]["splits"]}
 
     value = units_total / (ms_total_max * 1e-3) / 1e12
     flops_bwd_main = 10.0 * d * Hq * pairs
@@ -653,6 +666,7 @@ def main():
         "gpu_launches": ((8 if grad == B.GRAD_BF16 else 7) + (5 if args.reorder else 0)) * args.steps,
         "cpu_baseline": cpu_baseline,
         "per_config": per_config,
+        "rollout_decode": rollout_decode,
     }
     print(json.dumps(line), flush=True)
     D.shutdown()

@@ -778,7 +778,7 @@ __global__ void cache_evict_kernel(const int32_t* __restrict__ ranges, int n_ran
             const unsigned gm = __ballot_sync(0xffffffffu, valid && !keep);
             const unsigned lt = (1u << lane) - 1u;
             __syncwarp();
-            if (keep) bt[kept + __popc(km & lt)] = page;          // kept + rank <= i: never ahead of the reads of this round
+            if (keep) bt[kept + __popc(km & lt)] = page;          // kept + rank <= i: never ahead of the reads of this pass
             else if (valid) stack[base + fpos + __popc(gm & lt)] = page;
             kept += __popc(km);
             fpos += __popc(gm);
